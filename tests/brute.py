@@ -1,0 +1,101 @@
+"""Brute-force statements used to pin the oracle on tiny inputs (pure Python / numpy).
+
+Nothing here is shared with the oracle or the CUDA path: attention is the textbook
+full softmax over the explicitly retained list, hits come from enumerating subsets,
+CRF is the closed-form sum over a recorded hit log (Section 5.2), and eviction is an
+exhaustive argmin.
+"""
+from __future__ import annotations
+
+import itertools
+
+import numpy as np
+import torch
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    return t.to(torch.float64).numpy()
+
+
+def naive_attention(q, K, V, scale):
+    """q [G,d], K [n,d], V [n,d] float64 -> (prob [G,n], y [G,d])."""
+    s = scale * (q @ K.T)
+    s = s - s.max(axis=1, keepdims=True)
+    e = np.exp(s)
+    p = e / e.sum(axis=1, keepdims=True)
+    return p, p @ V
+
+
+def smallest_covering_sets(pbar, p):
+    """All subsets of minimum cardinality whose mass reaches p; [(mass, frozenset)]."""
+    n = len(pbar)
+    for r in range(1, n + 1):
+        found = []
+        for S in itertools.combinations(range(n), r):
+            m = float(sum(pbar[i] for i in S))
+            if m >= p:
+                found.append((m, frozenset(S)))
+        if found:
+            return found
+    return []
+
+
+def brute_hits(pbar, p):
+    """The hit set by enumeration: minimum cardinality, then maximum mass."""
+    found = smallest_covering_sets(pbar, p)
+    if not found:  # total mass below p (rounding): everything is needed
+        return frozenset(range(len(pbar))), 1
+    best = max(m for m, _ in found)
+    winners = [S for m, S in found if m == best]
+    return winners[0], len(winners)
+
+
+class BruteUnit:
+    """One (sequence, layer, kv-head) cache simulated from definitions."""
+
+    def __init__(self, budget, lam, top_p, scale):
+        self.B, self.lam, self.p, self.scale = budget, lam, top_p, scale
+        self.pos, self.K, self.V = [], [], []
+        self.hits = []     # per entry: list of hit times
+        self.arrival = []  # per entry: arrival time (tau before the first hit)
+
+    def append(self, pos, k, v, arrival):
+        self.pos.append(pos); self.K.append(k); self.V.append(v)
+        self.hits.append([]); self.arrival.append(arrival)
+
+    def crf(self, i, t):
+        """Closed form CRF(e_i) = sum_j lambda^(t - t_j) over the hit log."""
+        return sum(self.lam ** (t - tj) for tj in self.hits[i])  # 0 ** 0 == 1
+
+    def last(self, i):
+        return self.hits[i][-1] if self.hits[i] else self.arrival[i]
+
+    def step(self, q, t, track=True):
+        """Attention at time t; returns (y, min_gap) where min_gap is the smallest
+        relative distance of any decision from flipping (for skipping near-ties)."""
+        K, V = np.stack(self.K), np.stack(self.V)
+        prob, y = naive_attention(q, K, V, self.scale)
+        gap = np.inf
+        if track:
+            pbar = prob.mean(axis=0)
+            (S, nwin) = brute_hits(list(pbar), self.p)
+            srt = np.sort(pbar)[::-1]
+            c = np.cumsum(srt)
+            k = len(S)
+            gap = min(gap, abs(c[k - 1] - self.p), abs((c[k - 2] if k > 1 else 0.0) - self.p))
+            if k < len(srt):
+                gap = min(gap, abs(srt[k - 1] - srt[k]) / srt[k - 1])
+            for i in S:
+                self.hits[i].append(t)
+            n = len(self.pos)
+            if n > self.B:
+                keys = [(self.crf(i, t), self.last(i), self.pos[i], i) for i in range(n)]
+                keys.sort()
+                kk = n - self.B
+                a, b = keys[kk - 1][0], keys[kk][0]
+                if a != b:
+                    gap = min(gap, abs(b - a) / max(abs(a), abs(b)))
+                gone = {x[3] for x in keys[:kk]}
+                for name in ("pos", "K", "V", "hits", "arrival"):
+                    setattr(self, name, [x for j, x in enumerate(getattr(self, name)) if j not in gone])
+        return y, gap
