@@ -1,0 +1,172 @@
+/*
+ * crystalkv.h — C ABI of the Crystal-KV decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * One handle owns, on one GPU, the compressed KV cache of `batch` independent
+ * sequences of a GQA transformer: a slot-indexed K/V pool per sequence, per
+ * (sequence, layer, kv head) slot lists with CRF / last-hit-time metadata, and the
+ * per-head budgets.  Notation follows the paper: B budget, p top-p threshold, lambda
+ * CRF decay, t time step, tau last hit time, CRF the combined recency-frequency score.
+ *
+ * Conventions
+ *   - Tensors are dense, row-major, bf16 (2 bytes per element), head_dim = 128.
+ *   - "dev" pointers are device memory on the handle's GPU, "host" pointers are host
+ *     memory.  The caller owns every pointer it passes; the library owns the pool,
+ *     the lists and the metadata and frees them in crystalkv_destroy.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Work is enqueued on it; hot-path calls neither synchronise the host nor allocate.
+ *   - Every call returns 0 on success or a negative CRYSTALKV_E* code; nothing throws
+ *     or aborts across this boundary.  crystalkv_strerror() gives the text of a code,
+ *     crystalkv_last_error() the detail of the handle's most recent failure.
+ *   - A handle is not thread-safe and is used with one stream at a time.
+ */
+#ifndef CRYSTALKV_H
+#define CRYSTALKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CRYSTALKV_OK 0
+#define CRYSTALKV_EINVAL (-1)   /* null pointer, value out of range, unsupported dtype / head_dim */
+#define CRYSTALKV_ESTATE (-2)   /* call out of order, capacity or context exhausted */
+#define CRYSTALKV_ENOMEM (-3)   /* device allocation failed */
+#define CRYSTALKV_ECUDA (-4)    /* CUDA runtime error (sticky for the handle) */
+#define CRYSTALKV_ECHECK (-5)   /* a device-side consistency check raised the handle's error word */
+
+#define CRYSTALKV_BF16 1
+
+#define CRYSTALKV_MODE_EVICT 0   /* Algorithm 1 runs every think step */
+#define CRYSTALKV_MODE_FULLKV 1  /* FullKV baseline of Section 6.1: nothing tracked, nothing evicted */
+
+#define CRYSTALKV_STAGE_THINK 0
+#define CRYSTALKV_STAGE_ANSWER 1
+
+typedef struct crystalkv crystalkv_t;
+
+typedef struct {
+  int32_t n_layers;        /* L */
+  int32_t n_q_heads;       /* multiple of n_kv_heads; group size G = n_q_heads / n_kv_heads <= 8 */
+  int32_t n_kv_heads;      /* H */
+  int32_t head_dim;        /* 128 */
+  int32_t batch;           /* independent sequences, each with its own budgets (Algorithm 2 is per inference) */
+  int32_t dtype;           /* CRYSTALKV_BF16 */
+  int32_t budget_per_head; /* B_total per sequence = budget_per_head * L * H (Algorithm 2 input) */
+  int32_t min_budget;      /* floor of a head's budget under reallocation; 0 = max(16, budget_per_head / 8) */
+  int32_t max_budget;      /* cap of a head's budget; 0 = 4 * budget_per_head; >= budget_per_head */
+  int32_t max_answer_tokens; /* entries a head may append beyond its budget in the answer stage */
+  int32_t max_context;     /* largest token position + 1; sizes the lambda^D table and FullKV capacity */
+  float top_p;             /* hit threshold p in (0, 1]; 0 = 0.9 (Section 6.4) */
+  float lambda;            /* CRF decay in [0, 1]; negative = 0.6 (Section 6.4) */
+  float sm_scale;          /* logit scale; 0 = 1/sqrt(head_dim) */
+  int32_t mode;            /* CRYSTALKV_MODE_* */
+  int32_t device;          /* CUDA device ordinal */
+} crystalkv_config_t;
+
+/*
+ * Allocates the handle's device state (pool, lists, metadata, lambda^D table, split-K
+ * scratch).  Section 5: one cache per (layer, head) with CRF and tau per entry.
+ * Errors: EINVAL (bad field, *out untouched), ENOMEM, ECUDA.
+ */
+int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out);
+
+/* Frees everything the handle owns.  NULL is accepted. */
+int crystalkv_destroy(crystalkv_t* h);
+
+/*
+ * Loads a prompt into one layer (Algorithm 1 inputs K/V, Q^last) and runs one
+ * Algorithm 1 pass with Q^last at t = P-1, so CRF/tau are seeded and heads whose
+ * prompt exceeds their budget are evicted down to it.
+ *   k, v   dev  [batch][P][H][128]     q_last dev [batch][Hq][128] (query of token P-1)
+ * P must satisfy 1 <= P <= budget_per_head + max_answer_tokens (evict mode) or
+ * P < max_context (FullKV mode).  Errors: EINVAL; ESTATE if the layer was prefilled.
+ */
+int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v,
+                      const void* q_last, int P, void* stream);
+
+/*
+ * One decode step of one layer for all sequences (Section 2.2 attention fused with
+ * Algorithm 1): appends (k_new, v_new) at time t = previous t + 1, attends the G
+ * queries of every kv head over its cache, writes `out`, and in the think stage of
+ * evict mode marks the top-p hit entries, updates CRF/tau (steps 2-3) and evicts the
+ * lowest-CRF entry of every head that is over budget (step 4), reusing its slot.
+ *   q, out dev [batch][Hq][128]        k_new, v_new dev [batch][H][128]
+ * Errors: EINVAL; ESTATE before prefill or when t would reach max_context or a head
+ * would outgrow its capacity.
+ */
+int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* k_new,
+                          const void* v_new, void* out, void* stream);
+
+/*
+ * The same step with pinned HOST buffers: copies q, k_new, v_new to the device, runs
+ * the step and copies `out` back, all enqueued on `stream` (no host synchronisation).
+ */
+int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host,
+                               const void* k_new_host, const void* v_new_host, void* out_host,
+                               void* stream);
+
+/* Think stage: Algorithm 1 runs.  Answer stage: the think cache is frozen, new tokens
+ * are appended beyond the budget and attended, nothing is tracked or evicted. */
+int crystalkv_set_stage(crystalkv_t* h, int stage);
+
+/*
+ * Algorithm 2 (Section 5.3), per sequence: aggregates every head's CRF decayed to the
+ * time of the last step, recomputes integer budgets that sum to B_total, and makes
+ * heads whose budget shrank evict down to it; freed slots return to the sequence's
+ * free list for heads that grew.  All layers must be at the same time step.
+ * Errors: ESTATE (layers out of step, FullKV mode, before prefill).
+ */
+int crystalkv_rebudget(crystalkv_t* h, void* stream);
+
+/*
+ * Token positions retained by (layer, seq, kv_head), ascending, into host memory.
+ * Synchronises `stream`.  *n_out receives the count; ESTATE if cap is too small.
+ */
+int crystalkv_get_retained(crystalkv_t* h, int layer, int seq, int kv_head,
+                           int32_t* pos_out_host, int32_t cap, int32_t* n_out, void* stream);
+
+/* Current budgets, host int32 [batch][L][H].  Synchronises `stream`. */
+int crystalkv_get_budgets(crystalkv_t* h, int32_t* out_host, void* stream);
+
+/*
+ * Per-entry state of one head, sorted by position: records of three int32
+ * {position, CRF as fp32 bits, tau}.  host_buf holds cap records; *n receives the
+ * count.  Synchronises `stream`.
+ */
+int crystalkv_export_state(crystalkv_t* h, int layer, int seq, int kv_head, int32_t* host_buf,
+                           int32_t cap, int32_t* n, void* stream);
+
+/*
+ * Overwrites CRF and tau of the listed positions (records as in export).  Every
+ * position must be present in the head's cache (else ESTATE, nothing changed).
+ */
+int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head,
+                           const int32_t* host_buf, int32_t n, void* stream);
+
+/* Sets one head's budget directly (tests and checkpoint restore). */
+int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_t budget,
+                         void* stream);
+
+/* Time step of the layer's last completed step (P-1 after prefill, -1 before). */
+int crystalkv_time(crystalkv_t* h, int layer);
+
+/*
+ * Bytes the Section 2.2 / Algorithm 1 data flow must move for the steps run so far:
+ * *kv_bytes = sum over steps and heads of entries attended * 512 (K and V rows).
+ * Synchronises `stream`; counters are kept on the device and cost one atomic per head.
+ */
+int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t* hits,
+                           uint64_t* evictions, void* stream);
+
+/* Reads and clears the handle's device error word (0 = clean).  Synchronises `stream`. */
+int crystalkv_check(crystalkv_t* h, void* stream);
+
+const char* crystalkv_strerror(int code);
+const char* crystalkv_last_error(crystalkv_t* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CRYSTALKV_H */

@@ -51,7 +51,7 @@ typedef struct {
     int32_t pos;
     float crf;
     int32_t tau;
-    uint16_t *k, *v; /* bf16 bit patterns, head_dim each */
+    double *k, *v; /* the bf16 inputs converted exactly to fp64, head_dim each */
 } okv_entry;
 
 typedef struct {
@@ -98,10 +98,9 @@ static void unit_append(okv *o, okv_unit *u, int pos, const uint16_t *k, const u
     e->pos = pos;
     e->crf = crf;
     e->tau = tau;
-    e->k = (uint16_t *)malloc((size_t)d * 2);
-    e->v = (uint16_t *)malloc((size_t)d * 2);
-    memcpy(e->k, k, (size_t)d * 2);
-    memcpy(e->v, v, (size_t)d * 2);
+    e->k = (double *)malloc((size_t)d * sizeof(double));
+    e->v = (double *)malloc((size_t)d * sizeof(double));
+    for (int c = 0; c < d; ++c) { e->k[c] = bf16_to_double(k[c]); e->v[c] = bf16_to_double(v[c]); }
 }
 
 /* remove entry i, keeping the order of the others (a real compaction) */
@@ -129,31 +128,58 @@ static void log_tie(okv *o, int layer, int seq, int head, int t, int kind) {
 /*
  * AttnScore = softmax(q K^T), y = AttnScore V  (Section 2.2), for the G query heads
  * that share one KV head.  Reading: the logits carry a scale factor (1/sqrt(d) by
- * default); the paper's formula leaves it out.
- *   q: [G][d] bf16 bits; krows/vrows: n pointers to d bf16 bits.
- *   prob: [G][n] fp64 out; y: [G][d] fp64 out.
+ * default); the paper's formula leaves it out.  Every dot product and every output
+ * channel is summed in ascending index order; the G heads are only evaluated side by
+ * side.
+ *   q: [G][d]; krows/vrows: n pointers to d values; prob: [G][n] out; y: [G][d] out.
  */
-void okv_attention(const uint16_t *q, const uint16_t *const *krows, const uint16_t *const *vrows,
-                   int n, int G, int d, double scale, double *prob, double *y) {
+static void attention_f64(const double *q, const double *const *krows, const double *const *vrows,
+                          int n, int G, int d, double scale, double *prob, double *y) {
+    double s[64];
+    for (int i = 0; i < n; ++i) {
+        const double *k = krows[i];
+        for (int g = 0; g < G; ++g) s[g] = 0.0;
+        for (int c = 0; c < d; ++c)
+            for (int g = 0; g < G; ++g) s[g] += q[g * d + c] * k[c];
+        for (int g = 0; g < G; ++g) prob[(size_t)g * n + i] = scale * s[g];
+    }
     for (int g = 0; g < G; ++g) {
         double *p = prob + (size_t)g * n;
         double m = -INFINITY;
-        for (int i = 0; i < n; ++i) {
-            double s = 0.0;
-            for (int c = 0; c < d; ++c)
-                s += bf16_to_double(q[g * d + c]) * bf16_to_double(krows[i][c]);
-            p[i] = scale * s;
-            if (p[i] > m) m = p[i];
-        }
+        for (int i = 0; i < n; ++i) if (p[i] > m) m = p[i];
         double l = 0.0;
         for (int i = 0; i < n; ++i) { p[i] = exp(p[i] - m); l += p[i]; }
         for (int i = 0; i < n; ++i) p[i] /= l;
-        for (int c = 0; c < d; ++c) {
-            double acc = 0.0;
-            for (int i = 0; i < n; ++i) acc += p[i] * bf16_to_double(vrows[i][c]);
-            y[g * d + c] = acc;
+    }
+    for (int i = 0; i < G * d; ++i) y[i] = 0.0;
+    for (int i = 0; i < n; ++i) {
+        const double *v = vrows[i];
+        for (int g = 0; g < G; ++g) {
+            const double pi = prob[(size_t)g * n + i];
+            double *yg = y + (size_t)g * d;
+            for (int c = 0; c < d; ++c) yg[c] += pi * v[c];
         }
     }
+}
+
+/* the same from bf16 bit patterns: q [G][d], krows/vrows n pointers to d bf16 values */
+void okv_attention(const uint16_t *q, const uint16_t *const *krows, const uint16_t *const *vrows,
+                   int n, int G, int d, double scale, double *prob, double *y) {
+    double *qd = (double *)malloc((size_t)G * d * sizeof(double));
+    double *kv = (double *)malloc((size_t)2 * (n > 0 ? n : 1) * d * sizeof(double));
+    const double **kr = (const double **)malloc((size_t)(n > 0 ? n : 1) * sizeof(void *));
+    const double **vr = (const double **)malloc((size_t)(n > 0 ? n : 1) * sizeof(void *));
+    for (int i = 0; i < G * d; ++i) qd[i] = bf16_to_double(q[i]);
+    for (int i = 0; i < n; ++i) {
+        kr[i] = kv + (size_t)i * d;
+        vr[i] = kv + (size_t)(n + i) * d;
+        for (int c = 0; c < d; ++c) {
+            kv[(size_t)i * d + c] = bf16_to_double(krows[i][c]);
+            kv[(size_t)(n + i) * d + c] = bf16_to_double(vrows[i][c]);
+        }
+    }
+    attention_f64(qd, kr, vr, n, G, d, scale, prob, y);
+    free(qd); free(kv); free(kr); free(vr);
 }
 
 /* ------------------------------------------------------------------ Section 5.2: hits */
@@ -277,12 +303,15 @@ static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, i
                       int track, float *y) {
     okv_unit *u = unit_of(o, seq, layer, head);
     int n = u->n, d = o->c.head_dim, G = o->c.n_q_heads / o->c.n_kv_heads;
-    const uint16_t **kr = (const uint16_t **)malloc((size_t)n * sizeof(void *));
-    const uint16_t **vr = (const uint16_t **)malloc((size_t)n * sizeof(void *));
+    const double **kr = (const double **)malloc((size_t)n * sizeof(void *));
+    const double **vr = (const double **)malloc((size_t)n * sizeof(void *));
     for (int i = 0; i < n; ++i) { kr[i] = u->e[i].k; vr[i] = u->e[i].v; }
     double *prob = (double *)malloc((size_t)G * n * sizeof(double));
     double *yy = (double *)malloc((size_t)G * d * sizeof(double));
-    okv_attention(q, kr, vr, n, G, d, (double)o->c.sm_scale, prob, yy);
+    double *qd = (double *)malloc((size_t)G * d * sizeof(double));
+    for (int i = 0; i < G * d; ++i) qd[i] = bf16_to_double(q[i]);
+    attention_f64(qd, kr, vr, n, G, d, (double)o->c.sm_scale, prob, yy);
+    free(qd);
     if (y) for (int i = 0; i < G * d; ++i) y[i] = (float)yy[i];
     if (track) {
         double *pbar = (double *)malloc((size_t)n * sizeof(double));
@@ -310,7 +339,7 @@ static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, i
 
 okv *okv_create(const okv_config *c) {
     if (!c || c->n_layers < 1 || c->n_kv_heads < 1 || c->batch < 1 || c->head_dim < 1 ||
-        c->n_q_heads % c->n_kv_heads || c->max_context < 1)
+        c->n_q_heads % c->n_kv_heads || c->n_q_heads / c->n_kv_heads > 64 || c->max_context < 1)
         return NULL;
     okv *o = (okv *)calloc(1, sizeof(okv));
     o->c = *c;

@@ -1,0 +1,234 @@
+// Set-up and periodic kernels around the decode step: prompt insertion, Algorithm 2
+// (adaptive budget allocation) and the shrink pass that moves slot ownership between heads.
+#pragma once
+#include "common.cuh"
+#include "evict.cuh"
+
+namespace ckv {
+
+// ---------------------------------------------------------------------------------------
+// Prompt insertion for one layer: one CTA per (sequence, kv head).  Takes P + 1 slots from the
+// sequence's free list (P entries and the spare), copies the K/V rows into them and sets
+// pos = i, CRF = 0, tau = P - 1 (the time of the scoring pass that follows).
+//   k, v: [batch][P][H][128] bf16
+__global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int* n_out, int layer,
+                                                            const __nv_bfloat16* k,
+                                                            const __nv_bfloat16* v, int P) {
+  __shared__ int s_top;
+  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
+  const int uid = (seq * st.L + layer) * st.H + head;
+  const size_t mb = (size_t)uid * st.cap;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    int top = atomicSub(&st.free_top[seq], P + 1);
+    if (top < P + 1) {
+      atomicAdd(&st.free_top[seq], P + 1);
+      atomicOr(st.errword, ERR_FREE_UNDERFLOW);
+      top = -1;
+    }
+    s_top = top;
+  }
+  __syncthreads();
+  const int top = s_top;
+  if (top < 0) {
+    if (tid == 0) n_out[uid] = 0;
+    return;
+  }
+  const int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
+  for (int i = tid; i <= P; i += NT) {
+    st.list_slot[mb + i] = stack[top - 1 - i];
+    if (i < P) {
+      st.meta_pos[mb + i] = i;
+      st.meta_tau[mb + i] = P - 1;
+      st.meta_crf[mb + i] = 0.0f;
+    }
+  }
+  unsigned char* poolseq = st.pool + (size_t)seq * st.slots_per_seq * SLOT_BYTES;
+  const int piece = tid & 31;
+  for (int i = tid >> 5; i < P; i += NW) {
+    const int slot = stack[top - 1 - i];
+    const size_t off = (((size_t)seq * P + i) * st.H + head) * HD * 2;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(piece < 16 ? k : v) + off + (piece & 15) * 16;
+    *reinterpret_cast<uint4*>(poolseq + (size_t)slot * SLOT_BYTES + piece * 16) = *reinterpret_cast<const uint4*>(src);
+  }
+  if (tid == 0) n_out[uid] = P;
+}
+
+// ---------------------------------------------------------------------------------------
+// Algorithm 2 input: per head, the sum of CRF decayed to t_last over the retained entries,
+// each term truncated to 2^-32 fixed point so the sum does not depend on the order.
+__global__ void __launch_bounds__(NT) crf_sum_kernel(State st, const int* n_cur, int t_last,
+                                                     long long* Asum) {
+  __shared__ long long s_red[NW];
+  const int uid = blockIdx.x;
+  const size_t mb = (size_t)uid * st.cap;
+  const int n = n_cur[uid];
+  long long acc = 0;
+  for (int i = threadIdx.x; i < n; i += NT) {
+    const float d = __fmul_rn(st.tab[t_last - st.meta_tau[mb + i]], st.meta_crf[mb + i]);
+    acc += (long long)((double)d * 4294967296.0);
+  }
+  acc = (long long)warp_sum_u64((unsigned long long)acc);
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long tot = 0;
+    for (int x = 0; x < NW; ++x) tot += s_red[x];
+    Asum[uid] = tot;
+  }
+}
+
+// Block-wide: hand `extra` whole slots to the m heads listed in who[] in proportion to x[]:
+// floor of the real share, then one more each by largest fractional part (ties to the
+// lower head index).  Every fp64 operation is a single correctly rounded one, in the
+// order a sequential evaluation of the same formulas takes them.
+__device__ void share_out(long long extra, const int* who, int m, const double* x, long long* add,
+                          double* frac, int* order, double* s_d, long long* s_ll) {
+  const int tid = threadIdx.x;
+  if (m <= 0 || extra <= 0) return;
+  if (tid == 0) {
+    double W = 0.0;
+    for (int j = 0; j < m; ++j) W = __dadd_rn(W, x[who[j]]);
+    s_d[0] = W;
+  }
+  __syncthreads();
+  const double W = s_d[0];
+  long long given = 0;
+  for (int j = tid; j < m; j += NT) {
+    const int k = who[j];
+    const double xs = (W > 0.0) ? __ddiv_rn(__dmul_rn((double)extra, x[k]), W)
+                                : __ddiv_rn((double)extra, (double)m);
+    const double f = floor(xs);
+    add[k] += (long long)f;
+    given += (long long)f;
+    frac[j] = __dsub_rn(xs, f);
+  }
+  given = (long long)warp_sum_u64((unsigned long long)given);
+  if ((tid & 31) == 0) s_ll[tid >> 5] = given;
+  __syncthreads();
+  long long left = extra;
+  for (int w = 0; w < NW; ++w) left -= s_ll[w];
+  // rank of j under (frac descending, head index ascending)
+  for (int j = tid; j < m; j += NT) {
+    const double fj = frac[j];
+    const int kj = who[j];
+    int rank = 0;
+    for (int i = 0; i < m; ++i) rank += (frac[i] > fj) || (frac[i] == fj && who[i] < kj);
+    order[rank] = j;
+    if (left >= 0) add[kj] += left / m + (rank < (int)(left % m) ? 1 : 0);
+  }
+  __syncthreads();
+  if (left < 0 && tid == 0) {  // over-given by rounding: take back from the smallest fractions
+    for (long long j = m - 1; left < 0; --j) {
+      if (j < 0) j = m - 1;
+      const int k = who[order[j]];
+      if (add[k] > 0) { add[k] -= 1; ++left; }
+    }
+  }
+  __syncthreads();
+}
+
+// Algorithm 2, one CTA per sequence:
+//   eta_i = sum_j A_ij / sum_j B_ij,  B'_i = B_total eta_i / sum_i eta_i,
+//   eta_ij = A_ij / B_ij,             B'_ij = B'_i eta_ij / sum_j eta_ij,
+// integerised: min_b per head is set aside, the rule divides the remainder by largest
+// remainders so the budgets sum to B_total, heads above max_b are clamped and their excess
+// shared among the rest in the same proportions.  sum_i eta_i = 0 keeps the budgets.
+__global__ void __launch_bounds__(NT) alg2_kernel(const long long* Asum, int* budget, int L, int H,
+                                                  long long B_total, int min_b, int max_b) {
+  extern __shared__ __align__(16) unsigned char sm[];
+  const int N = L * H, tid = threadIdx.x;
+  double* a = reinterpret_cast<double*>(sm);
+  double* x = a + N;
+  double* frac = x + N;
+  double* eta_l = frac + N;
+  double* S_l = eta_l + L;
+  long long* add = reinterpret_cast<long long*>(S_l + L);
+  int* who = reinterpret_cast<int*>(add + N);
+  int* order = who + N;
+  __shared__ double s_d[2];
+  __shared__ long long s_ll[NW + 1];
+  __shared__ int s_red[NW + 1];
+  const size_t base = (size_t)blockIdx.x * N;
+  for (int k = tid; k < N; k += NT) {
+    a[k] = __ddiv_rn((double)Asum[base + k], 4294967296.0);
+    add[k] = 0;
+    who[k] = k;
+  }
+  __syncthreads();
+  for (int i = tid; i < L; i += NT) {
+    double sa = 0.0, sb = 0.0, sl = 0.0;
+    for (int j = 0; j < H; ++j) {
+      const double bij = (double)budget[base + i * H + j];
+      sa = __dadd_rn(sa, a[i * H + j]);
+      sb = __dadd_rn(sb, bij);
+      sl = __dadd_rn(sl, __ddiv_rn(a[i * H + j], bij));
+    }
+    eta_l[i] = __ddiv_rn(sa, sb);
+    S_l[i] = sl;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double S = 0.0;
+    for (int i = 0; i < L; ++i) S = __dadd_rn(S, eta_l[i]);
+    s_d[1] = S;
+  }
+  __syncthreads();
+  const double S = s_d[1];
+  if (!(S > 0.0)) return;
+  const long long R = B_total - (long long)N * min_b;
+  for (int k = tid; k < N; k += NT) {
+    const int i = k / H;
+    const double layer_share = __ddiv_rn(__dmul_rn((double)R, eta_l[i]), S);
+    const double head_part = (S_l[i] > 0.0)
+        ? __ddiv_rn(__ddiv_rn(a[k], (double)budget[base + k]), S_l[i])
+        : __ddiv_rn(1.0, (double)H);
+    x[k] = __dmul_rn(layer_share, head_part);
+  }
+  __syncthreads();
+  share_out(R, who, N, x, add, frac, order, s_d, s_ll);
+  for (;;) {
+    long long excess = 0;
+    for (int k = tid; k < N; k += NT) {
+      const long long b = (long long)min_b + add[k];
+      if (b > max_b) { excess += b - max_b; add[k] = (long long)max_b - min_b; }
+    }
+    excess = (long long)warp_sum_u64((unsigned long long)excess);
+    __syncthreads();
+    if ((tid & 31) == 0) s_ll[tid >> 5] = excess;
+    __syncthreads();
+    excess = 0;
+    for (int w = 0; w < NW; ++w) excess += s_ll[w];
+    __syncthreads();
+    if (excess == 0) break;
+    int m = 0;
+    for (int b0 = 0; b0 < N; b0 += NT) {   // ordered compaction of the heads still under the cap
+      const int k = b0 + tid;
+      const int flag = (k < N) && ((long long)min_b + add[k] < max_b);
+      int tot;
+      const int r = block_excl_scan(flag, s_red, tot);
+      if (flag) who[m + r] = k;
+      m += tot;
+    }
+    __syncthreads();
+    if (m == 0) break;
+    share_out(excess, who, m, x, add, frac, order, s_d, s_ll);
+  }
+  for (int k = tid; k < N; k += NT) budget[base + k] = (int)(min_b + add[k]);
+}
+
+// ---------------------------------------------------------------------------------------
+// Shrink pass for the heads of one layer (one CTA per head): a head holding more entries than
+// its budget drops its lowest (decayed CRF, tau, pos) entries; their slots, beyond one spare,
+// go back to the sequence's free list, from which heads that grew refill step by step.
+__global__ void __launch_bounds__(NT) shrink_kernel(State st, int* n_cur, int layer, int t_last,
+                                                    int* tmp, int tmp_stride) {
+  __shared__ int sh[300];
+  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
+  const int uid = (seq * st.L + layer) * st.H + head;
+  const int n = n_cur[uid], B = st.budget[uid];
+  if (n <= B || n < 2) return;
+  evict_many(st, n_cur, uid, seq, n, min(n - B, n - 1), t_last, true, sh, tmp + (size_t)u * tmp_stride);
+}
+
+}  // namespace ckv

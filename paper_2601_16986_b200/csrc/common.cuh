@@ -1,0 +1,143 @@
+// Shared definitions of the Crystal-KV CUDA path (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ckv {
+
+constexpr int HD = 128;             // head_dim
+constexpr int ROW_BYTES = 256;      // one K or V row, bf16
+constexpr int SLOT_BYTES = 512;     // pool slot = K row followed by V row
+constexpr int GRP = 16;             // keys per streamed group
+constexpr int NW = 4;               // warps per CTA
+constexpr int NT = NW * 32;
+constexpr int NSLOT = 2;            // ring depth per warp, in groups
+constexpr int K_REGION = GRP * ROW_BYTES;
+constexpr int V_STRIDE = ROW_BYTES + 16;   // padded so 8 rows hit 8 different 16-byte bank groups
+constexpr int V_REGION = GRP * V_STRIDE;
+constexpr int RING_SLOT_BYTES = K_REGION + V_REGION;
+constexpr int RING_BYTES = NW * NSLOT * RING_SLOT_BYTES;
+constexpr int GMIN = 4;             // fewest groups a working CTA takes
+constexpr int HIST_BINS = 2048;
+constexpr int MAX_UNITS_PER_CALL = 4096;
+
+// error word bits raised by device-side consistency checks (never a trap)
+constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence's free list was empty
+constexpr int ERR_OVER_EVICT = 2;       // a decode step found a head more than one entry over budget
+constexpr int ERR_CAPACITY = 4;         // a head's list would outgrow its capacity
+constexpr int ERR_NUCLEUS = 8;          // the top-p threshold search did not find its boundary
+
+struct State {
+  // K/V pool: [batch][slots_per_seq][512 B]
+  unsigned char* pool;
+  long long slots_per_seq;
+  int* free_stack;   // [batch][slots_per_seq]
+  int* free_top;     // [batch] number of free slots
+  // per unit (uid = (seq*L + layer)*H + head), capacity `cap` list positions
+  int* list_slot;    // [units][cap] slot of the entry at a list position; position n holds the spare
+  int* meta_pos;     // [units][cap] token position
+  int* meta_tau;     // [units][cap] last hit time
+  float* meta_crf;   // [units][cap] CRF at tau
+  int* nbuf[2];      // [2][units] entry counts, double buffered: a launch reads one and writes the other
+  int* budget;       // [units] == [batch][L][H]
+  const float* tab;  // lambda^D, D in [0, max_context]
+  int* errword;
+  unsigned long long* counters;  // entries attended, hits, evictions
+  int batch, L, H, cap;
+};
+
+// scratch shared by the launches of one handle (two sets, alternating per call)
+struct Scratch {
+  float* logits;     // [U][G][cap_s] scaled logits of the step
+  float* pbar;       // [U][cap_s] group-mean probabilities (reused as int scratch)
+  float* partials;   // [U][pmax][G*130] split-K partial (m, l, O)
+  int* ticket;       // [U]
+  int cap_s, pmax;
+};
+
+struct DecodeParams {
+  State st;
+  Scratch sc;
+  const __nv_bfloat16* q;       // [batch][Hq][128]
+  const __nv_bfloat16* k_new;   // [batch][H][128]
+  const __nv_bfloat16* v_new;
+  __nv_bfloat16* out;           // [batch][Hq][128]
+  const int* n_in;   // entry counts before this launch
+  int* n_out;        // entry counts after it (a different buffer: CTAs that start late still see n_in)
+  int layer;
+  int t;          // time of this step
+  int append;     // 1: decode (a new entry arrives); 0: scoring pass over the prompt
+  int track;      // 1: Algorithm 1 runs (hits, CRF, eviction)
+  int release;    // 1: freed slots beyond one spare go back to the free list (no pops in this launch)
+  float scale;    // logit scale
+  float scale_log2;
+  float top_p;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// ---- block-wide helpers (NT threads, `red` = NW*8 words of shared scratch) ----
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_sum_i(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Exclusive scan of one int per thread across the block; returns this thread's prefix and
+// the block total.  `red` needs NW+1 ints.  Contains two __syncthreads().
+__device__ __forceinline__ int block_excl_scan(int v, int* red, int& total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int x = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += x;
+  }
+  __syncthreads();
+  if (lane == 31) red[w] = inc;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    int x = red[i];
+    if (i < w) base += x;
+    tot += x;
+  }
+  total = tot;
+  return base + inc - v;
+}
+
+}  // namespace ckv

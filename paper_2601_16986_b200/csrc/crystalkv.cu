@@ -1,0 +1,577 @@
+// C ABI of the Crystal-KV decode hot path (see include/crystalkv.h).  Host code only
+// validates, keeps the per-layer clocks and launches; every step of the path runs in the
+// kernels of decode_kernel.cuh and aux_kernels.cuh.
+#include "../../include/crystalkv.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "aux_kernels.cuh"
+#include "decode_kernel.cuh"
+
+using namespace ckv;
+
+struct crystalkv {
+  crystalkv_config_t cfg;
+  int G = 0, U = 0, units = 0, cap = 0, num_sms = 0, grid = 0;
+  size_t smem = 0;
+  long long slots_per_seq = 0;
+  State st{};
+  Scratch sc[2]{};
+  int sc_idx = 0;
+  std::vector<int> t_layer, par;   // per layer: time of the last step, current count buffer
+  int stage = CRYSTALKV_STAGE_THINK;
+  int answer_steps = 0;
+  long long* Asum = nullptr;
+  __nv_bfloat16 *dq = nullptr, *dk = nullptr, *dv = nullptr, *dout = nullptr;  // staging for host I/O
+  __nv_bfloat16* dummy_out = nullptr;
+  float* tab = nullptr;
+  std::vector<void*> allocs;
+  std::string err;
+  bool cuda_dead = false;
+};
+
+namespace {
+
+thread_local std::string g_create_err;
+
+int fail(crystalkv_t* h, int code, const std::string& msg) {
+  if (h) h->err = msg;
+  return code;
+}
+
+#define CK(h, call)                                                                      \
+  do {                                                                                   \
+    cudaError_t e_ = (call);                                                             \
+    if (e_ != cudaSuccess) {                                                             \
+      if (h) (h)->cuda_dead = true;                                                      \
+      return fail((h), CRYSTALKV_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
+    }                                                                                    \
+  } while (0)
+
+template <typename T>
+int dalloc(crystalkv_t* h, T** p, size_t count) {
+  void* q = nullptr;
+  cudaError_t e = cudaMalloc(&q, std::max<size_t>(count, 1) * sizeof(T));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(h, e == cudaErrorMemoryAllocation ? CRYSTALKV_ENOMEM : CRYSTALKV_ECUDA,
+                std::string("cudaMalloc: ") + cudaGetErrorString(e));
+  }
+  h->allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return CRYSTALKV_OK;
+}
+
+__global__ void init_free_stack_kernel(int* stack, int* top, long long slots_per_seq, int batch) {
+  const long long total = slots_per_seq * batch;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i % slots_per_seq;
+    stack[i] = (int)(slots_per_seq - 1 - r);   // popping from the top hands out ascending slot ids
+  }
+  if (blockIdx.x == 0 && threadIdx.x < batch) top[threadIdx.x] = (int)slots_per_seq;
+  if (blockIdx.x == 0)
+    for (int b = threadIdx.x; b < batch; b += blockDim.x) top[b] = (int)slots_per_seq;
+}
+
+__global__ void fill_int_kernel(int* p, long long n, int v) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+    p[i] = v;
+}
+
+template <int G>
+cudaError_t prepare_decode(size_t smem, int* blocks_per_sm) {
+  cudaError_t e = cudaFuncSetAttribute(decode_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, decode_kernel<G>, NT, smem);
+}
+
+template <int G>
+cudaError_t launch_decode(const DecodeParams& p, int grid, size_t smem, cudaStream_t s) {
+  decode_kernel<G><<<grid, NT, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t prepare_dispatch(int G, size_t smem, int* bps) {
+  switch (G) {
+    case 1: return prepare_decode<1>(smem, bps);
+    case 2: return prepare_decode<2>(smem, bps);
+    case 3: return prepare_decode<3>(smem, bps);
+    case 4: return prepare_decode<4>(smem, bps);
+    case 5: return prepare_decode<5>(smem, bps);
+    case 6: return prepare_decode<6>(smem, bps);
+    case 7: return prepare_decode<7>(smem, bps);
+    case 8: return prepare_decode<8>(smem, bps);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_dispatch(int G, const DecodeParams& p, int grid, size_t smem, cudaStream_t s) {
+  switch (G) {
+    case 1: return launch_decode<1>(p, grid, smem, s);
+    case 2: return launch_decode<2>(p, grid, smem, s);
+    case 3: return launch_decode<3>(p, grid, smem, s);
+    case 4: return launch_decode<4>(p, grid, smem, s);
+    case 5: return launch_decode<5>(p, grid, smem, s);
+    case 6: return launch_decode<6>(p, grid, smem, s);
+    case 7: return launch_decode<7>(p, grid, smem, s);
+    case 8: return launch_decode<8>(p, grid, smem, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+int validate(const crystalkv_config_t* c, std::string& why) {
+  if (!c) { why = "cfg is NULL"; return CRYSTALKV_EINVAL; }
+  if (c->head_dim != HD) { why = "head_dim must be 128"; return CRYSTALKV_EINVAL; }
+  if (c->dtype != CRYSTALKV_BF16) { why = "dtype must be CRYSTALKV_BF16"; return CRYSTALKV_EINVAL; }
+  if (c->n_layers < 1 || c->n_kv_heads < 1 || c->batch < 1) { why = "n_layers, n_kv_heads, batch must be >= 1"; return CRYSTALKV_EINVAL; }
+  if (c->n_q_heads < c->n_kv_heads || c->n_q_heads % c->n_kv_heads) { why = "n_q_heads must be a multiple of n_kv_heads"; return CRYSTALKV_EINVAL; }
+  if (c->n_q_heads / c->n_kv_heads > 8) { why = "group size above 8"; return CRYSTALKV_EINVAL; }
+  if ((long long)c->batch * c->n_kv_heads > MAX_UNITS_PER_CALL) { why = "batch * n_kv_heads above 4096"; return CRYSTALKV_EINVAL; }
+  if (c->mode != CRYSTALKV_MODE_EVICT && c->mode != CRYSTALKV_MODE_FULLKV) { why = "bad mode"; return CRYSTALKV_EINVAL; }
+  if (c->max_context < 2) { why = "max_context must be >= 2"; return CRYSTALKV_EINVAL; }
+  if (c->mode == CRYSTALKV_MODE_EVICT && c->budget_per_head < 1) { why = "budget_per_head must be >= 1"; return CRYSTALKV_EINVAL; }
+  if (c->min_budget < 0 || c->max_budget < 0 || c->max_answer_tokens < 0) { why = "negative budget bound"; return CRYSTALKV_EINVAL; }
+  if (c->max_budget && c->max_budget < c->budget_per_head) { why = "max_budget below budget_per_head"; return CRYSTALKV_EINVAL; }
+  if (c->min_budget > c->budget_per_head) { why = "min_budget above budget_per_head"; return CRYSTALKV_EINVAL; }
+  if (c->top_p < 0.f || c->top_p > 1.f) { why = "top_p outside (0, 1]"; return CRYSTALKV_EINVAL; }
+  if (c->lambda > 1.f) { why = "lambda above 1"; return CRYSTALKV_EINVAL; }
+  if (c->sm_scale < 0.f) { why = "negative sm_scale"; return CRYSTALKV_EINVAL; }
+  if (c->device < 0) { why = "negative device"; return CRYSTALKV_EINVAL; }
+  return CRYSTALKV_OK;
+}
+
+int check_layer(crystalkv_t* h, int layer) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  if (layer < 0 || layer >= h->cfg.n_layers) return fail(h, CRYSTALKV_EINVAL, "layer out of range");
+  return CRYSTALKV_OK;
+}
+
+int check_unit(crystalkv_t* h, int layer, int seq, int head) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (seq < 0 || seq >= h->cfg.batch || head < 0 || head >= h->cfg.n_kv_heads)
+    return fail(h, CRYSTALKV_EINVAL, "seq or kv_head out of range");
+  return CRYSTALKV_OK;
+}
+
+DecodeParams make_params(crystalkv_t* h, int layer) {
+  DecodeParams p{};
+  p.st = h->st;
+  p.sc = h->sc[h->sc_idx];
+  h->sc_idx ^= 1;
+  p.layer = layer;
+  p.n_in = h->st.nbuf[h->par[layer]];
+  p.n_out = h->st.nbuf[h->par[layer] ^ 1];
+  p.scale = h->cfg.sm_scale;
+  p.scale_log2 = h->cfg.sm_scale * 1.44269504088896340736f;
+  p.top_p = h->cfg.top_p;
+  return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* crystalkv_strerror(int code) {
+  switch (code) {
+    case CRYSTALKV_OK: return "ok";
+    case CRYSTALKV_EINVAL: return "invalid argument";
+    case CRYSTALKV_ESTATE: return "call out of order or capacity exhausted";
+    case CRYSTALKV_ENOMEM: return "device allocation failed";
+    case CRYSTALKV_ECUDA: return "CUDA runtime error";
+    case CRYSTALKV_ECHECK: return "device-side consistency check failed";
+  }
+  return "unknown error";
+}
+
+const char* crystalkv_last_error(crystalkv_t* h) { return h ? h->err.c_str() : g_create_err.c_str(); }
+
+int crystalkv_destroy(crystalkv_t* h) {
+  if (!h) return CRYSTALKV_OK;
+  cudaSetDevice(h->cfg.device);
+  for (void* p : h->allocs) cudaFree(p);
+  delete h;
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
+  std::string why;
+  int rc = validate(cfg, why);
+  if (rc) { g_create_err = why; return rc; }
+  if (!out) { g_create_err = "out is NULL"; return CRYSTALKV_EINVAL; }
+  crystalkv_t* h = new (std::nothrow) crystalkv();
+  if (!h) return CRYSTALKV_ENOMEM;
+  h->cfg = *cfg;
+  crystalkv_config_t& c = h->cfg;
+  if (c.top_p == 0.f) c.top_p = 0.9f;
+  if (c.lambda < 0.f) c.lambda = 0.6f;
+  if (c.sm_scale == 0.f) c.sm_scale = (float)(1.0 / std::sqrt((double)c.head_dim));
+  if (c.min_budget == 0) c.min_budget = std::min(c.budget_per_head, std::max(16, c.budget_per_head / 8));
+  if (c.max_budget == 0) c.max_budget = 4 * c.budget_per_head;
+  const bool evict = c.mode == CRYSTALKV_MODE_EVICT;
+  h->G = c.n_q_heads / c.n_kv_heads;
+  h->U = c.batch * c.n_kv_heads;
+  h->units = h->U * c.n_layers;
+  // list positions per head: entries up to the largest budget plus the arriving one and the
+  // answer-stage tail, plus the spare; FullKV keeps every token
+  h->cap = evict ? c.max_budget + 1 + c.max_answer_tokens + 1 : c.max_context + 1;
+  h->slots_per_seq = (long long)c.n_layers * c.n_kv_heads *
+                     (evict ? (long long)c.budget_per_head + 1 + c.max_answer_tokens : (long long)c.max_context + 1);
+  if (h->slots_per_seq > 0x7fffffffLL) { g_create_err = "more than 2^31 slots per sequence"; delete h; return CRYSTALKV_EINVAL; }
+
+#define CREATE_FAIL(code_)                    \
+  do {                                        \
+    int c_ = (code_);                         \
+    g_create_err = h->err;                    \
+    crystalkv_destroy(h);                     \
+    return c_;                                \
+  } while (0)
+#define CKC(call)                                                              \
+  do {                                                                         \
+    cudaError_t e_ = (call);                                                   \
+    if (e_ != cudaSuccess) {                                                   \
+      h->err = std::string(#call) + ": " + cudaGetErrorString(e_);             \
+      CREATE_FAIL(CRYSTALKV_ECUDA);                                            \
+    }                                                                          \
+  } while (0)
+#define DA(ptr, count)                                   \
+  do {                                                   \
+    int r_ = dalloc(h, ptr, (size_t)(count));            \
+    if (r_) CREATE_FAIL(r_);                             \
+  } while (0)
+
+  CKC(cudaSetDevice(c.device));
+  cudaDeviceProp prop;
+  CKC(cudaGetDeviceProperties(&prop, c.device));
+  h->num_sms = prop.multiProcessorCount;
+  h->smem = RING_BYTES + (size_t)(h->U + 1) * sizeof(int);
+  int bps = 0;
+  CKC(prepare_dispatch(h->G, h->smem, &bps));
+  if (bps < 1) { h->err = "decode kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
+  h->grid = h->num_sms * bps;
+
+  State& st = h->st;
+  st.batch = c.batch; st.L = c.n_layers; st.H = c.n_kv_heads; st.cap = h->cap;
+  st.slots_per_seq = h->slots_per_seq;
+  DA(&st.pool, (size_t)c.batch * h->slots_per_seq * SLOT_BYTES);
+  DA(&st.free_stack, (size_t)c.batch * h->slots_per_seq);
+  DA(&st.free_top, c.batch);
+  DA(&st.list_slot, (size_t)h->units * h->cap);
+  DA(&st.meta_pos, (size_t)h->units * h->cap);
+  DA(&st.meta_tau, (size_t)h->units * h->cap);
+  DA(&st.meta_crf, (size_t)h->units * h->cap);
+  DA(&st.nbuf[0], h->units);
+  DA(&st.nbuf[1], h->units);
+  DA(&st.budget, h->units);
+  DA(&h->tab, (size_t)c.max_context + 1);
+  st.tab = h->tab;
+  DA(&st.errword, 1);
+  DA(&st.counters, 4);
+  DA(&h->Asum, h->units);
+  const int capgroups = (h->cap + GRP - 1) / GRP;
+  for (int i = 0; i < 2; ++i) {
+    Scratch& sc = h->sc[i];
+    sc.cap_s = evict ? h->cap : 1;
+    sc.pmax = capgroups / GMIN + 2;
+    DA(&sc.logits, (size_t)h->U * h->G * sc.cap_s);
+    DA(&sc.pbar, (size_t)h->U * sc.cap_s);
+    DA(&sc.partials, (size_t)h->U * sc.pmax * h->G * (HD + 2));
+    DA(&sc.ticket, h->U);
+    CKC(cudaMemset(sc.ticket, 0, (size_t)h->U * sizeof(int)));
+  }
+  const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
+  DA(&h->dq, qn); DA(&h->dout, qn); DA(&h->dk, kn); DA(&h->dv, kn); DA(&h->dummy_out, qn);
+
+  // lambda^D as fp32 from an fp64 pow; pow(0, 0) = 1 keeps same-step hits when lambda = 0
+  {
+    std::vector<float> tab((size_t)c.max_context + 1);
+    for (int D = 0; D <= c.max_context; ++D) tab[D] = (float)std::pow((double)c.lambda, (double)D);
+    CKC(cudaMemcpy(h->tab, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice));
+  }
+  init_free_stack_kernel<<<1024, 256>>>(st.free_stack, st.free_top, h->slots_per_seq, c.batch);
+  fill_int_kernel<<<256, 256>>>(st.budget, h->units, c.budget_per_head);
+  CKC(cudaMemset(st.nbuf[0], 0, (size_t)h->units * sizeof(int)));
+  CKC(cudaMemset(st.nbuf[1], 0, (size_t)h->units * sizeof(int)));
+  CKC(cudaMemset(st.errword, 0, sizeof(int)));
+  CKC(cudaMemset(st.counters, 0, 4 * sizeof(unsigned long long)));
+  CKC(cudaGetLastError());
+  CKC(cudaDeviceSynchronize());
+  h->t_layer.assign(c.n_layers, -1);
+  h->par.assign(c.n_layers, 0);
+  *out = h;
+  return CRYSTALKV_OK;
+#undef CREATE_FAIL
+#undef CKC
+#undef DA
+}
+
+int crystalkv_set_stage(crystalkv_t* h, int stage) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (stage != CRYSTALKV_STAGE_THINK && stage != CRYSTALKV_STAGE_ANSWER) return fail(h, CRYSTALKV_EINVAL, "bad stage");
+  if (stage == CRYSTALKV_STAGE_THINK && h->answer_steps > 0)
+    return fail(h, CRYSTALKV_ESTATE, "answer tokens were appended; the think stage cannot resume");
+  h->stage = stage;
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_time(crystalkv_t* h, int layer) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return -1;
+  return h->t_layer[layer];
+}
+
+int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v, const void* q_last,
+                      int P, void* stream) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!k || !v || !q_last) return fail(h, CRYSTALKV_EINVAL, "null tensor");
+  const crystalkv_config_t& c = h->cfg;
+  const bool evict = c.mode == CRYSTALKV_MODE_EVICT;
+  if (P < 1) return fail(h, CRYSTALKV_EINVAL, "P must be >= 1");
+  if (evict && P > c.budget_per_head + c.max_answer_tokens)
+    return fail(h, CRYSTALKV_EINVAL, "prompt longer than budget_per_head + max_answer_tokens");
+  if (P >= c.max_context) return fail(h, CRYSTALKV_EINVAL, "prompt reaches max_context");
+  if (h->t_layer[layer] >= 0) return fail(h, CRYSTALKV_ESTATE, "layer already prefilled");
+  CK(h, cudaSetDevice(c.device));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  prefill_insert_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer,
+                                            static_cast<const __nv_bfloat16*>(k),
+                                            static_cast<const __nv_bfloat16*>(v), P);
+  CK(h, cudaGetLastError());
+  if (evict) {
+    // one Algorithm 1 pass with Q^last at t = P-1: seeds CRF/tau, evicts down to the budget
+    DecodeParams p = make_params(h, layer);
+    p.q = static_cast<const __nv_bfloat16*>(q_last);
+    p.k_new = p.v_new = nullptr;
+    p.out = h->dummy_out;
+    p.t = P - 1;
+    p.append = 0; p.track = 1; p.release = 1;
+    CK(h, launch_dispatch(h->G, p, h->grid, h->smem, s));
+    h->par[layer] ^= 1;
+  }
+  h->t_layer[layer] = P - 1;
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* k_new,
+                          const void* v_new, void* out, void* stream) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!q || !k_new || !v_new || !out) return fail(h, CRYSTALKV_EINVAL, "null tensor");
+  const crystalkv_config_t& c = h->cfg;
+  if (h->t_layer[layer] < 0) return fail(h, CRYSTALKV_ESTATE, "decode before prefill");
+  const int t = h->t_layer[layer] + 1;
+  if (t >= c.max_context) return fail(h, CRYSTALKV_ESTATE, "max_context reached");
+  const bool track = c.mode == CRYSTALKV_MODE_EVICT && h->stage == CRYSTALKV_STAGE_THINK;
+  if (c.mode == CRYSTALKV_MODE_EVICT && h->stage == CRYSTALKV_STAGE_ANSWER) {
+    // every layer appends once per answer token; count tokens by layer 0's clock
+    const int used = h->answer_steps / c.n_layers;
+    if (used >= c.max_answer_tokens) return fail(h, CRYSTALKV_ESTATE, "max_answer_tokens reached");
+  }
+  DecodeParams p = make_params(h, layer);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.t = t;
+  p.append = 1; p.track = track ? 1 : 0; p.release = 0;
+  CK(h, launch_dispatch(h->G, p, h->grid, h->smem, static_cast<cudaStream_t>(stream)));
+  h->par[layer] ^= 1;
+  h->t_layer[layer] = t;
+  if (!track && c.mode == CRYSTALKV_MODE_EVICT) h->answer_steps++;
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host, const void* k_new_host,
+                               const void* v_new_host, void* out_host, void* stream) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!q_host || !k_new_host || !v_new_host || !out_host) return fail(h, CRYSTALKV_EINVAL, "null tensor");
+  const crystalkv_config_t& c = h->cfg;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t qb = (size_t)c.batch * c.n_q_heads * HD * 2, kb = (size_t)c.batch * c.n_kv_heads * HD * 2;
+  CK(h, cudaMemcpyAsync(h->dq, q_host, qb, cudaMemcpyHostToDevice, s));
+  CK(h, cudaMemcpyAsync(h->dk, k_new_host, kb, cudaMemcpyHostToDevice, s));
+  CK(h, cudaMemcpyAsync(h->dv, v_new_host, kb, cudaMemcpyHostToDevice, s));
+  rc = crystalkv_decode_step(h, layer, h->dq, h->dk, h->dv, h->dout, stream);
+  if (rc) return rc;
+  CK(h, cudaMemcpyAsync(out_host, h->dout, qb, cudaMemcpyDeviceToHost, s));
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_rebudget(crystalkv_t* h, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  const crystalkv_config_t& c = h->cfg;
+  if (c.mode != CRYSTALKV_MODE_EVICT) return fail(h, CRYSTALKV_ESTATE, "rebudget in FullKV mode");
+  const int t_last = h->t_layer[0], par = h->par[0];
+  if (t_last < 0) return fail(h, CRYSTALKV_ESTATE, "rebudget before prefill");
+  for (int l = 1; l < c.n_layers; ++l)
+    if (h->t_layer[l] != t_last || h->par[l] != par) return fail(h, CRYSTALKV_ESTATE, "layers are at different time steps");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int* n_cur = h->st.nbuf[par];
+  crf_sum_kernel<<<h->units, NT, 0, s>>>(h->st, n_cur, t_last, h->Asum);
+  CK(h, cudaGetLastError());
+  const int N = c.n_layers * c.n_kv_heads;
+  const size_t sm = (size_t)N * (3 * sizeof(double) + sizeof(long long) + 2 * sizeof(int)) + (size_t)c.n_layers * 2 * sizeof(double);
+  if (sm > 48 * 1024) CK(h, cudaFuncSetAttribute(alg2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+  const long long B_total = (long long)c.budget_per_head * N;
+  alg2_kernel<<<c.batch, NT, sm, s>>>(h->Asum, h->st.budget, c.n_layers, c.n_kv_heads, B_total, c.min_budget, c.max_budget);
+  CK(h, cudaGetLastError());
+  const Scratch& sc = h->sc[h->sc_idx];
+  for (int l = 0; l < c.n_layers; ++l) {
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, n_cur, l, t_last, reinterpret_cast<int*>(sc.pbar), sc.cap_s);
+    CK(h, cudaGetLastError());
+  }
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_t budget, void* stream) {
+  int rc = check_unit(h, layer, seq, kv_head);
+  if (rc) return rc;
+  const crystalkv_config_t& c = h->cfg;
+  if (c.mode != CRYSTALKV_MODE_EVICT) return fail(h, CRYSTALKV_ESTATE, "set_budget in FullKV mode");
+  if (budget < 1 || budget > c.max_budget) return fail(h, CRYSTALKV_EINVAL, "budget outside [1, max_budget]");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
+  CK(h, cudaMemcpyAsync(h->st.budget + uid, &budget, sizeof(int), cudaMemcpyHostToDevice, s));
+  CK(h, cudaStreamSynchronize(s));
+  if (h->t_layer[layer] >= 0) {
+    const Scratch& sc = h->sc[h->sc_idx];
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer, h->t_layer[layer],
+                                      reinterpret_cast<int*>(sc.pbar), sc.cap_s);
+    CK(h, cudaGetLastError());
+  }
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_get_budgets(crystalkv_t* h, int32_t* out_host, void* stream) {
+  if (!h || !out_host) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  CK(h, cudaMemcpyAsync(out_host, h->st.budget, (size_t)h->units * sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_export_state(crystalkv_t* h, int layer, int seq, int kv_head, int32_t* host_buf,
+                           int32_t cap, int32_t* n_out, void* stream) {
+  int rc = check_unit(h, layer, seq, kv_head);
+  if (rc) return rc;
+  if (!host_buf || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  const crystalkv_config_t& c = h->cfg;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
+  int n = 0;
+  CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  *n_out = n;
+  if (n > cap) return fail(h, CRYSTALKV_ESTATE, "buffer too small");
+  std::vector<int> pos(n), tau(n);
+  std::vector<float> crf(n);
+  const size_t mb = (size_t)uid * h->cap;
+  CK(h, cudaMemcpyAsync(pos.data(), h->st.meta_pos + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaMemcpyAsync(tau.data(), h->st.meta_tau + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaMemcpyAsync(crf.data(), h->st.meta_crf + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  std::vector<int> idx(n);
+  for (int i = 0; i < n; ++i) idx[i] = i;
+  std::sort(idx.begin(), idx.end(), [&](int a, int b) { return pos[a] < pos[b]; });
+  for (int i = 0; i < n; ++i) {
+    int32_t bits;
+    std::memcpy(&bits, &crf[idx[i]], 4);
+    host_buf[3 * i] = pos[idx[i]];
+    host_buf[3 * i + 1] = bits;
+    host_buf[3 * i + 2] = tau[idx[i]];
+  }
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_get_retained(crystalkv_t* h, int layer, int seq, int kv_head, int32_t* pos_out_host,
+                           int32_t cap, int32_t* n_out, void* stream) {
+  int rc = check_unit(h, layer, seq, kv_head);
+  if (rc) return rc;
+  if (!pos_out_host || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  const crystalkv_config_t& c = h->cfg;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
+  int n = 0;
+  CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  *n_out = n;
+  if (n > cap) return fail(h, CRYSTALKV_ESTATE, "buffer too small");
+  CK(h, cudaMemcpyAsync(pos_out_host, h->st.meta_pos + (size_t)uid * h->cap, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  std::sort(pos_out_host, pos_out_host + n);
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head, const int32_t* host_buf,
+                           int32_t n_rec, void* stream) {
+  int rc = check_unit(h, layer, seq, kv_head);
+  if (rc) return rc;
+  if (!host_buf || n_rec < 0) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  const crystalkv_config_t& c = h->cfg;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
+  int n = 0;
+  CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  std::vector<int> pos(n), tau(n);
+  std::vector<float> crf(n);
+  const size_t mb = (size_t)uid * h->cap;
+  CK(h, cudaMemcpyAsync(pos.data(), h->st.meta_pos + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaMemcpyAsync(tau.data(), h->st.meta_tau + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaMemcpyAsync(crf.data(), h->st.meta_crf + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  std::vector<std::pair<int, int>> where(n);
+  for (int i = 0; i < n; ++i) where[i] = {pos[i], i};
+  std::sort(where.begin(), where.end());
+  for (int r = 0; r < n_rec; ++r) {
+    auto it = std::lower_bound(where.begin(), where.end(), std::make_pair((int)host_buf[3 * r], -1));
+    if (it == where.end() || it->first != host_buf[3 * r]) return fail(h, CRYSTALKV_ESTATE, "position not in the cache");
+    std::memcpy(&crf[it->second], &host_buf[3 * r + 1], 4);
+    tau[it->second] = host_buf[3 * r + 2];
+  }
+  CK(h, cudaMemcpyAsync(h->st.meta_tau + mb, tau.data(), (size_t)n * 4, cudaMemcpyHostToDevice, s));
+  CK(h, cudaMemcpyAsync(h->st.meta_crf + mb, crf.data(), (size_t)n * 4, cudaMemcpyHostToDevice, s));
+  CK(h, cudaStreamSynchronize(s));
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t* hits,
+                           uint64_t* evictions, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned long long v[4];
+  CK(h, cudaMemcpyAsync(v, h->st.counters, sizeof(v), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  if (entries_attended) *entries_attended = v[0];
+  if (hits) *hits = v[1];
+  if (evictions) *evictions = v[2];
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_check(crystalkv_t* h, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int w = 0;
+  CK(h, cudaMemcpyAsync(&w, h->st.errword, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  if (w == 0) return CRYSTALKV_OK;
+  CK(h, cudaMemsetAsync(h->st.errword, 0, sizeof(int), s));
+  std::string msg = "device error word:";
+  if (w & ERR_FREE_UNDERFLOW) msg += " free-list underflow;";
+  if (w & ERR_OVER_EVICT) msg += " head more than one entry over budget in a decode step;";
+  if (w & ERR_CAPACITY) msg += " head list capacity exceeded;";
+  if (w & ERR_NUCLEUS) msg += " top-p boundary not found;";
+  return fail(h, CRYSTALKV_ECHECK, msg);
+}
+
+}  // extern "C"

@@ -1,0 +1,141 @@
+// Algorithm 1 step 4 as block-wide device routines: pick the k entries of a head that are
+// lowest under (CRF decayed to now, tau, position) and edit the head's slot list in place.
+// No K/V row is moved: a leaving entry's slot stays in the list past the live range as a
+// spare, and spares beyond one go back to the sequence's free list.
+#pragma once
+#include "common.cuh"
+
+namespace ckv {
+
+struct Key96 {
+  uint32_t w[3];  // CRF_temp bits (>= +0, so unsigned order == float order), tau, pos
+};
+
+__device__ __forceinline__ Key96 entry_key(const State& st, size_t mb, int i, int t) {
+  Key96 k;
+  const int tau = st.meta_tau[mb + i];
+  // lambda^(t - tau) * CRF, one fp32 rounding (Algorithm 1 steps 2-3 before the "+ 1")
+  k.w[0] = __float_as_uint(__fmul_rn(st.tab[t - tau], st.meta_crf[mb + i]));
+  k.w[1] = static_cast<uint32_t>(tau);
+  k.w[2] = static_cast<uint32_t>(st.meta_pos[mb + i]);
+  return k;
+}
+
+__device__ __forceinline__ bool key_le(const Key96& a, const uint32_t* b) {
+  if (a.w[0] != b[0]) return a.w[0] < b[0];
+  if (a.w[1] != b[1]) return a.w[1] < b[1];
+  return a.w[2] <= b[2];
+}
+
+// Moves entry `src` of a head into list position `dst` and leaves dst's slot at `src`.
+__device__ __forceinline__ void swap_into(const State& st, size_t mb, int dst, int src) {
+  const int freed = st.list_slot[mb + dst];
+  st.list_slot[mb + dst] = st.list_slot[mb + src];
+  st.meta_pos[mb + dst] = st.meta_pos[mb + src];
+  st.meta_tau[mb + dst] = st.meta_tau[mb + src];
+  st.meta_crf[mb + dst] = st.meta_crf[mb + src];
+  st.list_slot[mb + src] = freed;
+}
+
+// Spares at list positions (n_new, n_old) return to the sequence's free list; the one at
+// n_new stays with the head.  Only called from launches in which no head pops a slot.
+__device__ __forceinline__ void release_spares(const State& st, size_t mb, int seq, int n_new,
+                                               int n_old, int* s_base) {
+  const int cnt = n_old - n_new - 1;
+  if (cnt <= 0) return;
+  if (threadIdx.x == 0) *s_base = atomicAdd(&st.free_top[seq], cnt);
+  __syncthreads();
+  const int base = *s_base;
+  int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
+  for (int r = threadIdx.x; r < cnt; r += NT) stack[base + r] = st.list_slot[mb + n_new + 1 + r];
+  __syncthreads();
+}
+
+// Removes the k lowest entries (1 <= k < n) of head `uid` at time t.  `sh` is >= 1.2 KB of
+// shared scratch, `tmp` a global int scratch of >= n words.  All NT threads call it.
+__device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n, int k, int t,
+                           bool release, int* sh, int* tmp) {
+  const size_t mb = (size_t)uid * st.cap;
+  int* hist = sh;             // 256
+  int* s_kw = sh + 256;       // 3 words of the k-th key
+  int* s_krem = sh + 259;
+  int* red = sh + 260;        // NW + 1
+  const int tid = threadIdx.x;
+  if (tid < 3) s_kw[tid] = 0;
+  if (tid == 0) *s_krem = k;
+  __syncthreads();
+  // MSB-first radix select of the k-th smallest 96-bit key, 8 bits per pass
+  for (int word = 0; word < 3; ++word) {
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int b = tid; b < 256; b += NT) hist[b] = 0;
+      __syncthreads();
+      const uint32_t k0 = s_kw[0], k1 = s_kw[1], k2 = s_kw[2];
+      const uint32_t kw[3] = {k0, k1, k2};
+      for (int i = tid; i < n; i += NT) {
+        const Key96 key = entry_key(st, mb, i, t);
+        bool match = true;
+        for (int x = 0; x < word; ++x) match = match && (key.w[x] == kw[x]);
+        if (shift < 24) match = match && ((key.w[word] >> (shift + 8)) == (kw[word] >> (shift + 8)));
+        if (match) atomicAdd(&hist[(key.w[word] >> shift) & 255u], 1);
+      }
+      __syncthreads();
+      if (tid < 32) {
+        int loc = 0;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) loc += hist[tid * 8 + b];
+        int inc = loc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          int x = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += x;
+        }
+        const int krem = *s_krem;
+        const int before = inc - loc;
+        if (before < krem && krem <= inc) {  // exactly one lane
+          int cum = before;
+          for (int b = 0; b < 8; ++b) {
+            const int c = hist[tid * 8 + b];
+            if (cum + c >= krem) {
+              s_kw[word] = static_cast<int>(kw[word] | (static_cast<uint32_t>(tid * 8 + b) << shift));
+              *s_krem = krem - cum;
+              break;
+            }
+            cum += c;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  const uint32_t kth[3] = {(uint32_t)s_kw[0], (uint32_t)s_kw[1], (uint32_t)s_kw[2]};
+  const int nk = n - k;
+  // holes: leaving entries inside the surviving range [0, nk)
+  int run = 0;
+  for (int base = 0; base < nk; base += NT) {
+    const int i = base + tid;
+    const int flag = (i < nk) && key_le(entry_key(st, mb, i, t), kth);
+    int tot;
+    const int r = block_excl_scan(flag, red, tot);
+    if (flag) tmp[run + r] = i;
+    run += tot;
+  }
+  __syncthreads();
+  // movers: staying entries in the tail [nk, n) fill the holes in order
+  run = 0;
+  for (int base = nk; base < n; base += NT) {
+    const int i = base + tid;
+    const int flag = (i < n) && !key_le(entry_key(st, mb, i, t), kth);
+    int tot;
+    const int r = block_excl_scan(flag, red, tot);
+    if (flag) swap_into(st, mb, tmp[run + r], i);
+    run += tot;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    n_out[uid] = nk;
+    atomicAdd(&st.counters[2], (unsigned long long)k);
+  }
+  if (release) release_spares(st, mb, seq, nk, n, s_krem);
+}
+
+}  // namespace ckv
