@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Decode-step throughput of the Crystal-KV hot path on B200 (one JSON line on stdout).
+
+A step = one token through every layer: fused attention + LRFU update + eviction per
+layer, plus the adaptive budget reallocation every `rebudget_every` steps.  Default
+workload: the 14B-shaped configuration (48 layers, 40 q / 8 kv heads, batch 32, budget
+1024 per head, reallocation every 128 steps), synthetic seeded inputs.
+
+  python bench.py --gpus 1 --steps 256 --warmup 130
+  python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (replicas: batch sharded, no collective)
+  python bench.py --impl reference      (the CPU oracle, timed on the host cores)
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from synth import WORKLOADS  # noqa: E402
+
+METRIC = "decode steps/s (attn+LRFU+evict, all layers)"
+UNIT = "steps/s"
+
+
+def shard_batch(batch: int, rank: int, world: int):
+    """Sequences of a global batch owned by `rank` (contiguous, as even as possible)."""
+    base, extra = divmod(batch, world)
+    lo = rank * base + min(rank, extra)
+    return list(range(lo, lo + base + (1 if rank < extra else 0)))
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------
+def oracle_sample(wl, layers: int, steps: int):
+    """Times the CPU oracle, as it stands, on `layers` layers of the full batch for `steps`
+    decode steps after a prefill; returns (full-model steps/s, threads, description)."""
+    from oracle import Oracle, OracleConfig
+    sub = wl.scaled(n_layers=layers)
+    ctx = wl.prompt + steps + 2
+    o = Oracle(OracleConfig(n_layers=layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, batch=wl.batch,
+                            budget_per_head=wl.budget_per_head, max_context=ctx,
+                            min_budget=min(wl.budget_per_head, max(16, wl.budget_per_head // 8)),
+                            max_budget=4 * wl.budget_per_head, top_p=wl.top_p, lam=wl.lam))
+    for l in range(layers):
+        k, v = sub.prompt_kv(l)
+        o.prefill(l, k, v, sub.queries(l, [wl.prompt - 1])[:, 0])
+    inputs = [[sub.step_inputs(l, wl.prompt + s) for l in range(layers)] for s in range(steps)]
+    t0 = time.perf_counter()
+    for s in range(steps):
+        for l in range(layers):
+            o.decode_step(l, *inputs[s][l])
+    dt = time.perf_counter() - t0
+    o.close()
+    per_full_step = dt / steps * (wl.n_layers / layers)
+    threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    desc = (f"{steps} decode steps of {layers} of {wl.n_layers} layers, full batch {wl.batch}, after a "
+            f"{wl.prompt}-token prefill; scaled by {wl.n_layers}/{layers} to a whole step")
+    return 1.0 / per_full_step, threads, desc
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per = []
+    layers = 1
+    total = args.steps + args.warmup
+    from oracle import Oracle, OracleConfig  # noqa: F401  (fail early if the oracle cannot build)
+    # one bounded sample per "step": a single layer of the full batch
+    sub = wl.scaled(n_layers=layers)
+    from oracle import Oracle as O, OracleConfig as OC
+    o = O(OC(n_layers=layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, batch=wl.batch,
+             budget_per_head=wl.budget_per_head, max_context=wl.prompt + total + 2,
+             min_budget=min(wl.budget_per_head, max(16, wl.budget_per_head // 8)),
+             max_budget=4 * wl.budget_per_head, top_p=wl.top_p, lam=wl.lam))
+    k, v = sub.prompt_kv(0)
+    o.prefill(0, k, v, sub.queries(0, [wl.prompt - 1])[:, 0])
+    for s in range(total):
+        ins = sub.step_inputs(0, wl.prompt + s)
+        t0 = time.perf_counter()
+        o.decode_step(0, *ins)
+        if s >= args.warmup:
+            per.append(time.perf_counter() - t0)
+    o.close()
+    ms = sum(per) / len(per) * 1000.0 * wl.n_layers
+    value = 1000.0 / ms
+    threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    sample = (f"each step = 1 of {wl.n_layers} layers of the full batch {wl.batch} on the host cores, "
+              f"scaled by {wl.n_layers} to a whole step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "layers": wl.n_layers,
+                   "budget_per_head": wl.budget_per_head},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=130)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4_qwen14b", choices=sorted(WORKLOADS))
+    ap.add_argument("--batch", type=int, default=0, help="override the per-GPU batch")
+    ap.add_argument("--budget", type=int, default=0, help="override budget_per_head")
+    ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    if args.batch:
+        wl = wl.scaled(batch=args.batch)
+    if args.budget:
+        wl = wl.scaled(budget_per_head=args.budget, prompt=min(wl.prompt, args.budget))
+    if args.impl == "reference":
+        return run_reference(args, wl)
+    if args.warmup < 3:
+        raise SystemExit("--warmup must be at least 3")
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2601_16986_b200 import Config, CrystalKV
+    # replicas: every rank holds `batch` sequences of its own (weak scaling, no collective);
+    # ranks differ only in the sequence ids their inputs are drawn for
+    seqs = [rank * wl.batch + b for b in range(wl.batch)]
+    L, B, Hq, H, d = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    total = args.warmup + args.steps
+    n_e2e = max(0, args.e2e_steps)
+    ctx = wl.prompt + total + n_e2e + 2
+    kv = CrystalKV(Config(n_layers=L, n_q_heads=Hq, n_kv_heads=H, batch=B, budget_per_head=wl.budget_per_head,
+                          max_context=ctx, top_p=wl.top_p, lam=wl.lam, device=local))
+    with torch.no_grad():
+        for l in range(L):
+            k, v = wl.prompt_kv(l, seqs=seqs, device=dev)
+            kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], seqs=seqs, device=dev)[:, 0].contiguous())
+            del k, v
+        # all step inputs resident in HBM before the timed region: [steps][L][batch][heads][d]
+        pos = torch.arange(wl.prompt, wl.prompt + total + n_e2e)
+        Q = torch.empty(len(pos), L, B, Hq, d, dtype=torch.bfloat16, device=dev)
+        K = torch.empty(len(pos), L, B, H, d, dtype=torch.bfloat16, device=dev)
+        V = torch.empty(len(pos), L, B, H, d, dtype=torch.bfloat16, device=dev)
+        chunk = 64
+        for l in range(L):
+            for c0 in range(0, len(pos), chunk):
+                pp = pos[c0:c0 + chunk]
+                Q[c0:c0 + len(pp), l] = wl.queries(l, pp, seqs=seqs, device=dev).transpose(0, 1)
+                K[c0:c0 + len(pp), l] = wl.keys(l, pp, seqs=seqs, device=dev).transpose(0, 1)
+                V[c0:c0 + len(pp), l] = wl.values(l, pp, seqs=seqs, device=dev).transpose(0, 1)
+        OUT = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=dev)
+    torch.cuda.synchronize()
+    kv.check()
+
+    lib, h = kv.lib, kv._h
+    stream = torch.cuda.current_stream()
+    sp = C.c_void_p(stream.cuda_stream)
+    qp = [[C.c_void_p(Q[s, l].data_ptr()) for l in range(L)] for s in range(len(pos))]
+    kp = [[C.c_void_p(K[s, l].data_ptr()) for l in range(L)] for s in range(len(pos))]
+    vp = [[C.c_void_p(V[s, l].data_ptr()) for l in range(L)] for s in range(len(pos))]
+    op = [C.c_void_p(OUT[l].data_ptr()) for l in range(L)]
+    every = wl.rebudget_every
+    launches = {"n": 0}
+    rb_events = []
+
+    def one_step(s, timed):
+        for l in range(L):
+            rc = lib.crystalkv_decode_step(h, l, qp[s][l], kp[s][l], vp[s][l], op[l], sp)
+            if rc:
+                raise RuntimeError(f"decode_step failed: {rc}")
+        if timed:
+            launches["n"] += L
+        if every and (s + 1) % every == 0:
+            if timed:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            rc = lib.crystalkv_rebudget(h, sp)
+            if rc:
+                raise RuntimeError(f"rebudget failed: {rc}")
+            if timed:
+                e1.record(stream)
+                rb_events.append((e0, e1))
+                launches["n"] += 2 + L
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for s in range(args.warmup):
+        one_step(s, False)
+    barrier()
+    c0 = kv.get_counters()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        ev0.record(stream)
+        for s in range(args.warmup, total):
+            one_step(s, True)
+        ev1.record(stream)
+        barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+    c1 = kv.get_counters()
+    kv.check()
+    ms_rb = sum(a.elapsed_time(b) for a, b in rb_events)
+    ms_per_step = ms_total / args.steps
+    value = world * args.steps / (ms_total / 1000.0)
+
+    # roofline of the dominant kernel (the fused decode kernel): algorithmic bytes per launch
+    n_launch = args.steps * L
+    entries = c1["entries_attended"] - c0["entries_attended"]
+    hits = c1["hits"] - c0["hits"]
+    io_bytes = n_launch * (2 * B * Hq * d * 2 + 2 * B * H * d * 2)
+    algo_bytes = entries * (512 + 4 + 8) + hits * 8 + io_bytes
+    kernel_ms = (ms_total - ms_rb) / n_launch
+    achieved = algo_bytes / n_launch / (kernel_ms / 1000.0) / 1e9
+    peak, peak_kind = measured_peaks()
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
+                "kernel": "decode_kernel", "launch_us": kernel_ms * 1000.0,
+                "algorithmic_bytes_per_launch": algo_bytes / n_launch,
+                "entries_per_launch": entries / n_launch, "hit_fraction": hits / max(entries, 1)}
+    traffic_file = os.path.join(ROOT, "profiles", "decode_kernel_traffic.json")
+    if os.path.exists(traffic_file):
+        with open(traffic_file) as f:
+            tj = json.load(f)
+        roofline["traffic"] = tj.get("dram_bytes_per_entry", 0) * entries / n_launch or None
+
+    # end to end: the same steps through the host-buffer entry point, copies inside the timed region
+    e2e = None
+    if n_e2e:
+        hq = [[Q[total + s, l].cpu().pin_memory() for l in range(L)] for s in range(n_e2e)]
+        hk = [[K[total + s, l].cpu().pin_memory() for l in range(L)] for s in range(n_e2e)]
+        hv = [[V[total + s, l].cpu().pin_memory() for l in range(L)] for s in range(n_e2e)]
+        ho = [torch.empty(B, Hq, d, dtype=torch.bfloat16).pin_memory() for l in range(L)]
+        hp = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        f0.record(stream)
+        for s in range(n_e2e):
+            for l in range(L):
+                rc = lib.crystalkv_decode_step_host(h, l, hp(hq[s][l]), hp(hk[s][l]), hp(hv[s][l]), hp(ho[l]), sp)
+                if rc:
+                    raise RuntimeError(f"decode_step_host failed: {rc}")
+            if every and (total + s + 1) % every == 0:
+                lib.crystalkv_rebudget(h, sp)
+        f1.record(stream)
+        barrier()
+        wall = time.perf_counter() - t0
+        ms_e = max_over_ranks(max(f0.elapsed_time(f1), wall * 1000.0), world, dev)
+        e2e = {"value": world * n_e2e / (ms_e / 1000.0), "unit": UNIT,
+               "h2d_bytes_per_step": L * (B * Hq * d * 2 + 2 * B * H * d * 2),
+               "d2h_bytes_per_step": L * B * Hq * d * 2, "steps": n_e2e}
+        kv.check()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v_cpu, threads, desc = oracle_sample(wl, layers=1, steps=4)
+        cpu = {"value": v_cpu, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "batch_per_gpu": B, "layers": L, "q_heads": Hq, "kv_heads": H,
+                       "head_dim": d, "budget_per_head": wl.budget_per_head, "prompt": wl.prompt,
+                       "rebudget_every": every, "top_p": wl.top_p, "lambda": wl.lam,
+                       "l2": "per-step working set (cache of all layers) far larger than L2; no flush",
+                       "parallelism": f"replicas x{world}, no collective"},
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches["n"],
+            "roofline": roofline, "cpu_baseline": cpu,
+            "rebudget_ms_in_timed_region": ms_rb,
+        }))
+    kv.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

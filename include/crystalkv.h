@@ -163,6 +163,15 @@ int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t*
 /* Reads and clears the handle's device error word (0 = clean).  Synchronises `stream`. */
 int crystalkv_check(crystalkv_t* h, void* stream);
 
+/*
+ * Debug check of slot ownership (the in-place slot reuse of Algorithm 1 step 4 and the
+ * slot hand-over of the reallocation): every pool slot of every sequence must be held
+ * exactly once, by the sequence's free list or by one head (entries plus one spare).
+ * Allocates a temporary, synchronises `stream`; not for the hot path.  ECHECK on failure,
+ * ESTATE before every layer is prefilled.
+ */
+int crystalkv_validate(crystalkv_t* h, void* stream);
+
 const char* crystalkv_strerror(int code);
 const char* crystalkv_last_error(crystalkv_t* h);
 

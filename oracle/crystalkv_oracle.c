@@ -604,8 +604,24 @@ int okv_get_budgets(okv *o, int32_t *out) { /* [batch][L][H] */
     return OKV_OK;
 }
 
+/*
+ * Sets one head's budget by hand; a head holding more than its new budget evicts down
+ * to it at once, exactly as after a reallocation (lowest CRF decayed to the time of the
+ * last step first).
+ */
 int okv_set_budget(okv *o, int layer, int seq, int head, int budget) {
-    unit_of(o, seq, layer, head)->budget = budget;
+    okv_unit *u = unit_of(o, seq, layer, head);
+    int t_last = o->t_layer[layer];
+    u->budget = budget;
+    if (t_last >= 0 && u->n > budget) {
+        float *ct = (float *)malloc((size_t)u->n * sizeof(float));
+        for (int i = 0; i < u->n; ++i) {
+            volatile float dcrf = o->tab[t_last - u->e[i].tau] * u->e[i].crf;
+            ct[i] = dcrf;
+        }
+        if (evict_lowest(u, ct, u->n - budget, o->c.tie_eps)) log_tie(o, layer, seq, head, t_last, OKV_TIE_EVICT);
+        free(ct);
+    }
     return OKV_OK;
 }
 

@@ -90,6 +90,7 @@ def load_library():
     lib.crystalkv_time.argtypes = [vp, i32]
     lib.crystalkv_get_counters.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
     lib.crystalkv_check.argtypes = [vp, vp]
+    lib.crystalkv_validate.argtypes = [vp, vp]
     lib.crystalkv_strerror.argtypes = [i32]
     lib.crystalkv_strerror.restype = C.c_char_p
     lib.crystalkv_last_error.argtypes = [vp]
@@ -216,3 +217,6 @@ class CrystalKV:
 
     def check(self):
         self._ck(self.lib.crystalkv_check(self._h, _stream()))
+
+    def validate(self):
+        self._ck(self.lib.crystalkv_validate(self._h, _stream()))

@@ -231,4 +231,38 @@ __global__ void __launch_bounds__(NT) shrink_kernel(State st, int* n_cur, int la
   evict_many(st, n_cur, uid, seq, n, min(n - B, n - 1), t_last, true, sh, tmp + (size_t)u * tmp_stride);
 }
 
+// ---------------------------------------------------------------------------------------
+// Consistency check of slot ownership: every pool slot of a sequence must be owned exactly
+// once, either by the free list or by one head (its n entries and its spare).
+__global__ void mark_free_kernel(State st, int* seen) {
+  const int seq = blockIdx.y;
+  const int top = st.free_top[seq];
+  const int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < top; i += (long long)gridDim.x * blockDim.x) {
+    const int s = stack[i];
+    if (s < 0 || s >= st.slots_per_seq) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);
+    else atomicAdd(&seen[(size_t)seq * st.slots_per_seq + s], 1);
+  }
+}
+
+__global__ void mark_owned_kernel(State st, const int* n_cur, int layer, int* seen) {
+  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
+  const int uid = (seq * st.L + layer) * st.H + head;
+  const size_t mb = (size_t)uid * st.cap;
+  const int n = n_cur[uid];
+  for (int i = threadIdx.x; i <= n; i += blockDim.x) {   // position n is the spare
+    const int s = st.list_slot[mb + i];
+    if (s < 0 || s >= st.slots_per_seq) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);
+    else atomicAdd(&seen[(size_t)seq * st.slots_per_seq + s], 1);
+  }
+}
+
+__global__ void count_bad_kernel(const int* seen, long long total, int* bad) {
+  int loc = 0;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x)
+    loc += (seen[i] != 1);
+  loc = warp_sum_i(loc);
+  if ((threadIdx.x & 31) == 0 && loc) atomicAdd(bad, loc);
+}
+
 }  // namespace ckv

@@ -558,6 +558,35 @@ int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t*
   return CRYSTALKV_OK;
 }
 
+int crystalkv_validate(crystalkv_t* h, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  const crystalkv_config_t& c = h->cfg;
+  for (int l = 0; l < c.n_layers; ++l)
+    if (h->t_layer[l] < 0) return fail(h, CRYSTALKV_ESTATE, "validate before every layer is prefilled");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const long long total = (long long)c.batch * h->slots_per_seq;
+  int* seen = nullptr;
+  CK(h, cudaMalloc(&seen, (size_t)(total + 2) * sizeof(int)));
+  cudaError_t e = cudaMemsetAsync(seen, 0, (size_t)(total + 2) * sizeof(int), s);
+  if (e == cudaSuccess) {
+    mark_free_kernel<<<dim3(256, c.batch), 256, 0, s>>>(h->st, seen);
+    for (int l = 0; l < c.n_layers; ++l)
+      mark_owned_kernel<<<h->U, 128, 0, s>>>(h->st, h->st.nbuf[h->par[l]], l, seen);
+    count_bad_kernel<<<1024, 256, 0, s>>>(seen, total, seen + total + 1);
+    e = cudaGetLastError();
+  }
+  int res[2] = {0, 0};
+  if (e == cudaSuccess) e = cudaMemcpyAsync(res, seen + total, 2 * sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  cudaFree(seen);
+  CK(h, e);
+  if (res[0] || res[1])
+    return fail(h, CRYSTALKV_ECHECK, "slot ownership broken: " + std::to_string(res[0]) + " ids out of range, " +
+                                         std::to_string(res[1]) + " slots not owned exactly once");
+  return CRYSTALKV_OK;
+}
+
 int crystalkv_check(crystalkv_t* h, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

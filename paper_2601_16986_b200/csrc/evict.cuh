@@ -37,11 +37,12 @@ __device__ __forceinline__ void swap_into(const State& st, size_t mb, int dst, i
   st.list_slot[mb + src] = freed;
 }
 
-// Spares at list positions (n_new, n_old) return to the sequence's free list; the one at
-// n_new stays with the head.  Only called from launches in which no head pops a slot.
+// Spares at list positions (n_new, n_old] return to the sequence's free list (the k freed
+// slots and the head's previous spare at n_old, minus the one at n_new that stays with the
+// head).  Only called from launches in which no head pops a slot.
 __device__ __forceinline__ void release_spares(const State& st, size_t mb, int seq, int n_new,
                                                int n_old, int* s_base) {
-  const int cnt = n_old - n_new - 1;
+  const int cnt = n_old - n_new;
   if (cnt <= 0) return;
   if (threadIdx.x == 0) *s_base = atomicAdd(&st.free_top[seq], cnt);
   __syncthreads();
@@ -51,7 +52,8 @@ __device__ __forceinline__ void release_spares(const State& st, size_t mb, int s
   __syncthreads();
 }
 
-// Removes the k lowest entries (1 <= k < n) of head `uid` at time t.  `sh` is >= 1.2 KB of
+// Removes the k lowest entries (1 <= k < n) of head `uid` at time t.  With `release` the head
+// must own a spare at list position n (true between steps and after prompt insertion).  `sh` is >= 1.2 KB of
 // shared scratch, `tmp` a global int scratch of >= n words.  All NT threads call it.
 __device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n, int k, int t,
                            bool release, int* sh, int* tmp) {

@@ -1,0 +1,239 @@
+"""GPU <-> oracle parity through the C ABI (needs a B200; run with -m gpu).
+
+Retained sets / CRF bits / tau must be bit-exact except where the oracle logged a tie
+(decision within 1e-6 relative of flipping); attention outputs within max-abs 2e-2 of the
+fp32 oracle output.  Full-size shapes are run with the whole batch on the GPU and whole
+sampled sequences on the oracle.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from synth import WORKLOADS, Workload
+from tests.harness import LockStep
+
+pytestmark = pytest.mark.gpu
+SCALE = float(os.environ.get("CRYSTALKV_TEST_SCALE", "1.0"))   # lengthen or shorten the sampled runs
+
+
+def steps(n):
+    return max(8, int(n * SCALE))
+
+
+def test_cfg1_every_step_of_the_full_run():
+    """Config 1 exactly: 256-token prompt, 2048 think steps, budget 512, state compared every step."""
+    wl = WORKLOADS["cfg1_gqa4_b512"]
+    ls = LockStep(wl, [0])
+    ls.prefill()
+    ls.compare()
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    r = ls.rep
+    print(f"cfg1: steps={r.steps} heads_compared={r.heads_compared} ties_logged={r.ties_logged} "
+          f"tie_explained={r.tie_explained} unexplained={len(r.unexplained)} max_out_err={r.max_out_err:.3e}")
+    ls.assert_clean()
+    for h in range(2):
+        assert len(ls.gpu.get_retained(0, 0, h)) == 512
+    c = ls.gpu.get_counters()
+    assert c["evictions"] == 2 * (256 + 2048 - 512)
+    ls.close()
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_every_group_size_with_ragged_tails(G):
+    """Budgets and prompts that are not multiples of the 16-key group; prompt above the
+    budget (prefill evicts many at once); several tiles per head."""
+    wl = Workload(name=f"g{G}", seed=100 + G, n_layers=2, n_q_heads=2 * G, n_kv_heads=2, batch=3,
+                  prompt=83, think_steps=70, budget_per_head=53, outlier="flat", outlier_frac=0.05)
+    ls = LockStep(wl, [0, 2], max_answer_tokens=40)
+    ls.prefill()
+    ls.compare()
+    for s in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert ls.rep.heads_compared > 0 and len(ls.gpu.get_retained(1, 2, 1)) == 53
+    ls.close()
+
+
+class _PairedKeys(Workload):
+    """Keys of positions 2i and 2i+1 are identical: exact ties in the group-mean probability."""
+
+    def keys(self, layer, positions, seqs=None, device="cpu"):
+        pos = (torch.as_tensor(positions, dtype=torch.int64) // 2) * 2
+        return super().keys(layer, pos, seqs, device)
+
+
+def test_equal_scores_take_the_earlier_position():
+    wl = _PairedKeys(name="pairs", seed=5, n_layers=1, n_q_heads=4, n_kv_heads=2, batch=2, prompt=40,
+                     think_steps=120, budget_per_head=48, top_p=0.6)
+    ls = LockStep(wl, [0, 1])
+    ls.prefill()
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
+@pytest.mark.parametrize("lam,top_p", [(0.0, 0.9), (1.0, 0.9), (0.6, 1.0), (0.6, 0.5), (0.3, 0.05)])
+def test_limits_of_lambda_and_p(lam, top_p):
+    """lambda = 0 (LRU), lambda = 1 (LFU), p = 1 (every entry is a hit) and small p."""
+    wl = Workload(name="lim", seed=31, n_layers=1, n_q_heads=4, n_kv_heads=1, batch=2, prompt=30,
+                  think_steps=150, budget_per_head=64, lam=lam, top_p=top_p)
+    ls = LockStep(wl, [0, 1])
+    ls.prefill()
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
+def test_rebudget_small_with_answer_stage():
+    """Adaptive reallocation every 16 steps on a small model, then an answer stage."""
+    wl = Workload(name="rb", seed=77, n_layers=3, n_q_heads=8, n_kv_heads=4, batch=3, prompt=64,
+                  think_steps=160, answer_steps=12, budget_per_head=64, rebudget_every=16,
+                  outlier="perhead", outlier_lo=0.01, outlier_hi=0.3)
+    ls = LockStep(wl, [0, 1, 2], max_answer_tokens=16)
+    ls.prefill()
+    for s in range(wl.think_steps):
+        ls.step()
+        if (s + 1) % wl.rebudget_every == 0:
+            ls.rebudget()
+    b = ls.gpu.get_budgets()
+    assert (b.reshape(3, -1).sum(axis=1) == 64 * 12).all() and b.min() >= 16 and b.max() <= 256
+    assert (b != 64).any()
+    ls.set_stage_answer()
+    for s in range(wl.answer_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert ls.rep.budgets_compared == 30
+    ls.close()
+
+
+def test_fullkv_mode_is_plain_decode_attention():
+    wl = Workload(name="full", seed=9, n_layers=2, n_q_heads=10, n_kv_heads=2, batch=2, prompt=100,
+                  think_steps=60, budget_per_head=16)
+    ls = LockStep(wl, [0, 1], mode=1)
+    ls.prefill()
+    for _ in range(wl.think_steps):
+        ls.step(compare_state=False)
+    ls.compare()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert len(ls.gpu.get_retained(1, 1, 1)) == 160
+    ls.close()
+
+
+def test_shrinking_one_budget_by_hand():
+    """set_budget below the current length evicts many at once and frees their slots."""
+    wl = Workload(name="sb", seed=12, n_layers=1, n_q_heads=2, n_kv_heads=2, batch=1, prompt=50,
+                  think_steps=30, budget_per_head=60)
+    ls = LockStep(wl, [0])
+    ls.prefill()
+    for _ in range(20):
+        ls.step()
+    ls.gpu.set_budget(0, 0, 1, 17)
+    ls.ora.set_budget(0, 0, 1, 17)
+    ls.compare()                   # both sides evict down at once
+    assert len(ls.gpu.get_retained(0, 0, 1)) == 17
+    ls.step()
+    for _ in range(9):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
+# ------------------------------------------------------------------ full-size shapes, sampled
+def _run_sampled(name, sample, n_steps, cmp_every, answer=0, max_answer=0):
+    wl = WORKLOADS[name]
+    wl = wl.scaled(think_steps=n_steps, answer_steps=answer)
+    ls = LockStep(wl, sample, max_answer_tokens=max_answer)
+    ls.prefill()
+    ls.compare()
+    for s in range(n_steps):
+        ls.step(compare_state=((s + 1) % cmp_every == 0))
+        if wl.rebudget_every and (s + 1) % wl.rebudget_every == 0:
+            ls.rebudget()
+    ls.compare()
+    if answer:
+        ls.set_stage_answer()
+        for _ in range(answer):
+            ls.step(compare_state=False)
+        ls.compare()
+    ls.gpu.check()
+    r = ls.rep
+    print(f"{name}: sampled seqs {sample}, steps={r.steps} heads_compared={r.heads_compared} "
+          f"ties_logged={r.ties_logged} tie_explained={r.tie_explained} unexplained={len(r.unexplained)} "
+          f"budgets_compared={r.budgets_compared} max_out_err={r.max_out_err:.3e}")
+    ls.assert_clean()
+    return ls
+
+
+def test_cfg2_qwen7b_shape_sampled():
+    """7B shape (28 layers, 28q/4kv, batch 8, budget 1024): past the point where heads fill."""
+    ls = _run_sampled("cfg2_qwen7b", [0, 7], steps(560), 40)
+    assert len(ls.gpu.get_retained(27, 7, 3)) == 1024
+    ls.close()
+
+
+def test_cfg3_llama8b_shape_sampled():
+    """8B shape (32 layers, 32q/8kv, batch 16, B_total = 2048 x heads), reallocation every 128."""
+    ls = _run_sampled("cfg3_llama8b", [15], steps(384), 32)
+    b = ls.gpu.get_budgets()
+    assert (b.reshape(16, -1).sum(axis=1) == 2048 * 32 * 8).all()
+    ls.close()
+
+
+def test_cfg4_qwen14b_shape_sampled():
+    """14B shape (48 layers, 40q/8kv, batch 32, B_total = 1024 x heads), reallocation every 128,
+    then answer steps: the configuration the bench times."""
+    ls = _run_sampled("cfg4_qwen14b", [31], steps(384), 32, answer=4, max_answer=8)
+    b = ls.gpu.get_budgets()
+    assert (b.reshape(32, -1).sum(axis=1) == 1024 * 48 * 8).all() and (b != 1024).any()
+    ls.close()
+
+
+def test_cfg5_sweep_cells_sampled():
+    """Two cells of the 14B sweep (fewer layers: the layers are independent without
+    reallocation): small budget with a long prompt, and a large budget."""
+    for batch, budget, prompt, n in [(8, 256, 200, steps(120)), (1, 4096, 4000, steps(150))]:
+        wl = WORKLOADS["cfg5_sweep14b"].scaled(n_layers=4, batch=batch, budget_per_head=budget,
+                                               prompt=prompt, think_steps=n)
+        ls = LockStep(wl, [batch - 1])
+        ls.prefill()
+        for s in range(n):
+            ls.step(compare_state=((s + 1) % 30 == 0))
+        ls.compare()
+        ls.gpu.check()
+        ls.assert_clean()
+        assert len(ls.gpu.get_retained(3, batch - 1, 7)) == budget
+        ls.close()
+
+
+# ------------------------------------------------------------------ error paths on a live handle
+def test_call_order_errors():
+    from paper_2601_16986_b200 import Config, CrystalKV, CrystalKVError
+    kv = CrystalKV(Config(n_layers=2, n_q_heads=4, n_kv_heads=2, batch=1, budget_per_head=32, max_context=64))
+    q = torch.zeros(1, 4, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(CrystalKVError) as e:
+        kv.decode_step(0, q, k, k)
+    assert e.value.code == -2
+    pk = torch.zeros(1, 8, 2, 128, dtype=torch.bfloat16, device="cuda")
+    kv.prefill(0, pk, pk, q)
+    with pytest.raises(CrystalKVError):
+        kv.prefill(0, pk, pk, q)              # twice
+    with pytest.raises(CrystalKVError):
+        kv.rebudget()                         # layer 1 not prefilled: layers out of step
+    with pytest.raises(CrystalKVError):
+        kv.decode_step(5, q, k, k)            # bad layer
+    kv.decode_step(0, q, k, k)
+    kv.check()
+    kv.close()
