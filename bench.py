@@ -185,6 +185,7 @@ def main():
     ap.add_argument("--workload", default="cfg4_qwen14b", choices=sorted(WORKLOADS))
     ap.add_argument("--batch", type=int, default=0, help="override the per-GPU batch")
     ap.add_argument("--budget", type=int, default=0, help="override budget_per_head")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")
     ap.add_argument("--e2e-steps", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -193,6 +194,8 @@ def main():
         wl = wl.scaled(batch=args.batch)
     if args.budget:
         wl = wl.scaled(budget_per_head=args.budget, prompt=min(wl.prompt, args.budget))
+    if args.layers:
+        wl = wl.scaled(n_layers=args.layers)
     if args.impl == "reference":
         return run_reference(args, wl)
     if args.warmup < 3:
