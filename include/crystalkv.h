@@ -14,6 +14,8 @@
  *     the lists and the metadata and frees them in crystalkv_destroy.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     Work is enqueued on it; hot-path calls neither synchronise the host nor allocate.
+ *     The Algorithm 1 part of a decode step runs on a stream the handle owns, ordered
+ *     behind the step's attention by an event; later calls order themselves behind it.
  *   - Every call returns 0 on success or a negative CRYSTALKV_E* code; nothing throws
  *     or aborts across this boundary.  crystalkv_strerror() gives the text of a code,
  *     crystalkv_last_error() the detail of the handle's most recent failure.
@@ -106,6 +108,15 @@ int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* 
 int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host,
                                const void* k_new_host, const void* v_new_host, void* out_host,
                                void* stream);
+
+/*
+ * Makes `stream` wait (on the device, without blocking the host) for all work the handle
+ * has enqueued on its internal stream: the Algorithm 1 kernels of earlier decode steps,
+ * which run behind the attention kernels so that they overlap the next layer.  `out` of
+ * a decode step never needs this; every call that reads or edits the cache state does it
+ * by itself.  Use it before recording an event that should cover whole steps.
+ */
+int crystalkv_join(crystalkv_t* h, void* stream);
 
 /* Think stage: Algorithm 1 runs.  Answer stage: the think cache is frozen, new tokens
  * are appended beyond the budget and attended, nothing is tracked or evicted. */

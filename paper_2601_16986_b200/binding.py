@@ -81,6 +81,7 @@ def load_library():
     lib.crystalkv_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.crystalkv_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.crystalkv_set_stage.argtypes = [vp, i32]
+    lib.crystalkv_join.argtypes = [vp, vp]
     lib.crystalkv_rebudget.argtypes = [vp, vp]
     lib.crystalkv_get_retained.argtypes = [vp, i32, i32, i32, vp, C.c_int32, p32, vp]
     lib.crystalkv_get_budgets.argtypes = [vp, vp, vp]
@@ -172,6 +173,9 @@ class CrystalKV:
                                                      C.c_void_p(k_new.data_ptr()), C.c_void_p(v_new.data_ptr()),
                                                      C.c_void_p(out.data_ptr()), _stream()))
         return out
+
+    def join(self):
+        self._ck(self.lib.crystalkv_join(self._h, _stream()))
 
     def set_stage(self, stage):
         self._ck(self.lib.crystalkv_set_stage(self._h, stage))

@@ -9,18 +9,16 @@ namespace ckv {
 constexpr int HD = 128;             // head_dim
 constexpr int ROW_BYTES = 256;      // one K or V row, bf16
 constexpr int SLOT_BYTES = 512;     // pool slot = K row followed by V row
-constexpr int GRP = 16;             // keys per streamed group
-constexpr int NW = 4;               // warps per CTA
+constexpr int GRP = 16;             // keys per streamed group (one MMA tile of keys)
+constexpr int NW = 8;               // warps per CTA
 constexpr int NT = NW * 32;
-constexpr int NSLOT = 2;            // ring depth per warp, in groups
-constexpr int K_REGION = GRP * ROW_BYTES;
-constexpr int V_STRIDE = ROW_BYTES + 16;   // padded so 8 rows hit 8 different 16-byte bank groups
-constexpr int V_REGION = GRP * V_STRIDE;
-constexpr int RING_SLOT_BYTES = K_REGION + V_REGION;
-constexpr int RING_BYTES = NW * NSLOT * RING_SLOT_BYTES;
-constexpr int GMIN = 4;             // fewest groups a working CTA takes
-constexpr int HIST_BINS = 2048;
+constexpr int STAGES = 3;           // ring depth per warp, in groups
+constexpr int STAGE_BYTES = GRP * SLOT_BYTES;          // K tile (4 KB) then V tile (4 KB), 16-byte chunks swizzled
+constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;  // 192 KB
+constexpr int GMIN = 4;             // fewest groups a working warp takes
+constexpr int QH = 8;               // query heads of a group as padded for the MMA N dimension
 constexpr int MAX_UNITS_PER_CALL = 4096;
+constexpr int NSETS = 3;            // scratch sets cycled by consecutive launches
 
 // error word bits raised by device-side consistency checks (never a trap)
 constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence's free list was empty
@@ -39,7 +37,7 @@ struct State {
   int* meta_pos;     // [units][cap] token position
   int* meta_tau;     // [units][cap] last hit time
   float* meta_crf;   // [units][cap] CRF at tau
-  int* nbuf[2];      // [2][units] entry counts, double buffered: a launch reads one and writes the other
+  int* nbuf[2];      // [2][units] entry counts, double buffered: a step reads one and writes the other
   int* budget;       // [units] == [batch][L][H]
   const float* tab;  // lambda^D, D in [0, max_context]
   int* errword;
@@ -47,11 +45,12 @@ struct State {
   int batch, L, H, cap;
 };
 
-// scratch shared by the launches of one handle (two sets, alternating per call)
+// scratch of one launch pair (attention kernel, then LRFU kernel); NSETS sets are cycled
 struct Scratch {
-  float* logits;     // [U][G][cap_s] scaled logits of the step
+  float* logits;     // [U][cap_s][QH] scaled logits of the step, one 32-byte row per entry
   float* pbar;       // [U][cap_s] group-mean probabilities (reused as int scratch)
-  float* partials;   // [U][pmax][G*130] split-K partial (m, l, O)
+  float* partials;   // [U][pmax][16 + G*128] split-K partial: m[8], l[8], O[G][128]
+  float* mfin;       // [U][QH] merged running maximum (log2 domain) per query head
   int* ticket;       // [U]
   int cap_s, pmax;
 };
@@ -63,12 +62,13 @@ struct DecodeParams {
   const __nv_bfloat16* k_new;   // [batch][H][128]
   const __nv_bfloat16* v_new;
   __nv_bfloat16* out;           // [batch][Hq][128]
-  const int* n_in;   // entry counts before this launch
-  int* n_out;        // entry counts after it (a different buffer: CTAs that start late still see n_in)
+  const int* n_in;   // entry counts before this step
+  int* n_out;        // entry counts after it
   int layer;
+  int G;          // query heads per kv head
   int t;          // time of this step
   int append;     // 1: decode (a new entry arrives); 0: scoring pass over the prompt
-  int track;      // 1: Algorithm 1 runs (hits, CRF, eviction)
+  int track;      // 1: Algorithm 1 runs (hits, CRF, eviction) in the LRFU kernel that follows
   int release;    // 1: freed slots beyond one spare go back to the free list (no pops in this launch)
   float scale;    // logit scale
   float scale_log2;
@@ -91,10 +91,8 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// ---- block-wide helpers (NT threads, `red` = NW*8 words of shared scratch) ----
+// ---- block-wide helpers (NT threads) ----
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -138,6 +136,25 @@ __device__ __forceinline__ int block_excl_scan(int v, int* red, int& total) {
   }
   total = tot;
   return base + inc - v;
+}
+
+// A head keeps its length and takes a fresh spare slot for list position n (decode steps in
+// which nothing left the head).  One thread calls it.
+__device__ __forceinline__ void keep_and_refill(const State& st, int* n_out, int uid, int seq, int n,
+                                                bool append) {
+  n_out[uid] = n;
+  if (!append) return;
+  if (n + 1 > st.cap) {
+    atomicOr(st.errword, ERR_CAPACITY);
+    return;
+  }
+  const int idx = atomicSub(&st.free_top[seq], 1) - 1;
+  if (idx < 0) {
+    atomicAdd(&st.free_top[seq], 1);
+    atomicOr(st.errword, ERR_FREE_UNDERFLOW);
+  } else {
+    st.list_slot[(size_t)uid * st.cap + n] = st.free_stack[(size_t)seq * st.slots_per_seq + idx];
+  }
 }
 
 }  // namespace ckv

@@ -1,6 +1,13 @@
 // C ABI of the Crystal-KV decode hot path (see include/crystalkv.h).  Host code only
 // validates, keeps the per-layer clocks and launches; every step of the path runs in the
-// kernels of decode_kernel.cuh and aux_kernels.cuh.
+// kernels of attn_kernel.cuh, lrfu_kernel.cuh and aux_kernels.cuh.
+//
+// Stream plan of a tracked decode step of layer l: the attention kernel runs on the caller's
+// stream (so `out` is ready in stream order), the LRFU kernel of the same layer on an
+// internal stream behind an event, which lets it overlap the attention kernel of the next
+// layer.  Before an attention kernel reuses a scratch set, or touches a layer whose LRFU
+// kernel of the previous step may still run, the caller's stream waits on that kernel's
+// event.  Everything else (prefill, reallocation, inspection) first joins the internal stream.
 #include "../../include/crystalkv.h"
 
 #include <algorithm>
@@ -11,8 +18,9 @@
 #include <string>
 #include <vector>
 
+#include "attn_kernel.cuh"
 #include "aux_kernels.cuh"
-#include "decode_kernel.cuh"
+#include "lrfu_kernel.cuh"
 
 using namespace ckv;
 
@@ -22,9 +30,14 @@ struct crystalkv {
   size_t smem = 0;
   long long slots_per_seq = 0;
   State st{};
-  Scratch sc[2]{};
-  int sc_idx = 0;
+  Scratch sc[NSETS]{};
   std::vector<int> t_layer, par;   // per layer: time of the last step, current count buffer
+  // LRFU launches are numbered; launch k uses scratch set k % NSETS and event k % EV_RING
+  static constexpr int EV_RING = 8;
+  cudaStream_t side = nullptr;
+  cudaEvent_t evA = nullptr, evF[EV_RING] = {};
+  long long kF = 0, joined = -1;
+  std::vector<long long> lastF;    // per layer: number of its latest LRFU launch, -1 = none
   int stage = CRYSTALKV_STAGE_THINK;
   int answer_steps = 0;
   long long* Asum = nullptr;
@@ -86,42 +99,21 @@ __global__ void fill_int_kernel(int* p, long long n, int v) {
 }
 
 template <int G>
-cudaError_t prepare_decode(size_t smem, int* blocks_per_sm) {
-  cudaError_t e = cudaFuncSetAttribute(decode_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, decode_kernel<G>, NT, smem);
-}
-
-template <int G>
-cudaError_t launch_decode(const DecodeParams& p, int grid, size_t smem, cudaStream_t s) {
-  decode_kernel<G><<<grid, NT, smem, s>>>(p);
+cudaError_t launch_lrfu(const DecodeParams& p, int grid, cudaStream_t s) {
+  lrfu_kernel<G><<<grid, NT, 0, s>>>(p);
   return cudaGetLastError();
 }
 
-cudaError_t prepare_dispatch(int G, size_t smem, int* bps) {
+cudaError_t lrfu_dispatch(int G, const DecodeParams& p, int grid, cudaStream_t s) {
   switch (G) {
-    case 1: return prepare_decode<1>(smem, bps);
-    case 2: return prepare_decode<2>(smem, bps);
-    case 3: return prepare_decode<3>(smem, bps);
-    case 4: return prepare_decode<4>(smem, bps);
-    case 5: return prepare_decode<5>(smem, bps);
-    case 6: return prepare_decode<6>(smem, bps);
-    case 7: return prepare_decode<7>(smem, bps);
-    case 8: return prepare_decode<8>(smem, bps);
-  }
-  return cudaErrorInvalidValue;
-}
-
-cudaError_t launch_dispatch(int G, const DecodeParams& p, int grid, size_t smem, cudaStream_t s) {
-  switch (G) {
-    case 1: return launch_decode<1>(p, grid, smem, s);
-    case 2: return launch_decode<2>(p, grid, smem, s);
-    case 3: return launch_decode<3>(p, grid, smem, s);
-    case 4: return launch_decode<4>(p, grid, smem, s);
-    case 5: return launch_decode<5>(p, grid, smem, s);
-    case 6: return launch_decode<6>(p, grid, smem, s);
-    case 7: return launch_decode<7>(p, grid, smem, s);
-    case 8: return launch_decode<8>(p, grid, smem, s);
+    case 1: return launch_lrfu<1>(p, grid, s);
+    case 2: return launch_lrfu<2>(p, grid, s);
+    case 3: return launch_lrfu<3>(p, grid, s);
+    case 4: return launch_lrfu<4>(p, grid, s);
+    case 5: return launch_lrfu<5>(p, grid, s);
+    case 6: return launch_lrfu<6>(p, grid, s);
+    case 7: return launch_lrfu<7>(p, grid, s);
+    case 8: return launch_lrfu<8>(p, grid, s);
   }
   return cudaErrorInvalidValue;
 }
@@ -162,18 +154,52 @@ int check_unit(crystalkv_t* h, int layer, int seq, int head) {
   return CRYSTALKV_OK;
 }
 
-DecodeParams make_params(crystalkv_t* h, int layer) {
+DecodeParams make_params(crystalkv_t* h, int layer, int set) {
   DecodeParams p{};
   p.st = h->st;
-  p.sc = h->sc[h->sc_idx];
-  h->sc_idx ^= 1;
+  p.sc = h->sc[set];
   p.layer = layer;
+  p.G = h->G;
   p.n_in = h->st.nbuf[h->par[layer]];
   p.n_out = h->st.nbuf[h->par[layer] ^ 1];
   p.scale = h->cfg.sm_scale;
   p.scale_log2 = h->cfg.sm_scale * 1.44269504088896340736f;
   p.top_p = h->cfg.top_p;
   return p;
+}
+
+// Makes `s` wait for every LRFU kernel launched so far.
+int join_side(crystalkv_t* h, cudaStream_t s) {
+  if (h->kF > 0) CK(h, cudaStreamWaitEvent(s, h->evF[(h->kF - 1) % crystalkv::EV_RING], 0));
+  h->joined = h->kF - 1;
+  return CRYSTALKV_OK;
+}
+
+// One attention launch on `s` and, when Algorithm 1 runs, its LRFU launch on the internal stream.
+int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
+  const bool track = p.track != 0;
+  const long long k = h->kF;
+  if (track) {
+    // launch k reuses the scratch of launch k - NSETS and continues the state its layer's
+    // previous LRFU launch wrote; the internal stream runs in order, so one event covers both
+    const long long need = std::max(k - NSETS, h->lastF[layer]);
+    if (need >= 0 && need > h->joined) {
+      CK(h, cudaStreamWaitEvent(s, h->evF[need % crystalkv::EV_RING], 0));
+      h->joined = need;
+    }
+    p.sc = h->sc[k % NSETS];
+  }
+  attn_kernel<<<h->grid, NT, h->smem, s>>>(p);
+  CK(h, cudaGetLastError());
+  if (track) {
+    CK(h, cudaEventRecord(h->evA, s));
+    CK(h, cudaStreamWaitEvent(h->side, h->evA, 0));
+    CK(h, lrfu_dispatch(h->G, p, h->U, h->side));
+    CK(h, cudaEventRecord(h->evF[k % crystalkv::EV_RING], h->side));
+    h->lastF[layer] = k;
+    h->kF = k + 1;
+  }
+  return CRYSTALKV_OK;
 }
 
 }  // namespace
@@ -197,6 +223,11 @@ const char* crystalkv_last_error(crystalkv_t* h) { return h ? h->err.c_str() : g
 int crystalkv_destroy(crystalkv_t* h) {
   if (!h) return CRYSTALKV_OK;
   cudaSetDevice(h->cfg.device);
+  cudaDeviceSynchronize();
+  if (h->side) cudaStreamDestroy(h->side);
+  if (h->evA) cudaEventDestroy(h->evA);
+  for (cudaEvent_t e : h->evF)
+    if (e) cudaEventDestroy(e);
   for (void* p : h->allocs) cudaFree(p);
   delete h;
   return CRYSTALKV_OK;
@@ -252,11 +283,15 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   cudaDeviceProp prop;
   CKC(cudaGetDeviceProperties(&prop, c.device));
   h->num_sms = prop.multiProcessorCount;
-  h->smem = RING_BYTES + (size_t)(h->U + 1) * sizeof(int);
+  h->smem = RING_BYTES + (size_t)(2 * h->U + 1) * sizeof(int);
   int bps = 0;
-  CKC(prepare_dispatch(h->G, h->smem, &bps));
-  if (bps < 1) { h->err = "decode kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
+  CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem));
+  CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
+  if (bps < 1) { h->err = "attention kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
   h->grid = h->num_sms * bps;
+  CKC(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
+  CKC(cudaEventCreateWithFlags(&h->evA, cudaEventDisableTiming));
+  for (cudaEvent_t& e : h->evF) CKC(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
 
   State& st = h->st;
   st.batch = c.batch; st.L = c.n_layers; st.H = c.n_kv_heads; st.cap = h->cap;
@@ -277,13 +312,14 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   DA(&st.counters, 4);
   DA(&h->Asum, h->units);
   const int capgroups = (h->cap + GRP - 1) / GRP;
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < NSETS; ++i) {
     Scratch& sc = h->sc[i];
     sc.cap_s = evict ? h->cap : 1;
     sc.pmax = capgroups / GMIN + 2;
-    DA(&sc.logits, (size_t)h->U * h->G * sc.cap_s);
+    DA(&sc.logits, (size_t)h->U * sc.cap_s * QH);
     DA(&sc.pbar, (size_t)h->U * sc.cap_s);
-    DA(&sc.partials, (size_t)h->U * sc.pmax * h->G * (HD + 2));
+    DA(&sc.partials, (size_t)h->U * sc.pmax * (16 + h->G * HD));
+    DA(&sc.mfin, (size_t)h->U * QH);
     DA(&sc.ticket, h->U);
     CKC(cudaMemset(sc.ticket, 0, (size_t)h->U * sizeof(int)));
   }
@@ -306,6 +342,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   CKC(cudaDeviceSynchronize());
   h->t_layer.assign(c.n_layers, -1);
   h->par.assign(c.n_layers, 0);
+  h->lastF.assign(c.n_layers, -1);
   *out = h;
   return CRYSTALKV_OK;
 #undef CREATE_FAIL
@@ -318,6 +355,7 @@ int crystalkv_set_stage(crystalkv_t* h, int stage) {
   if (stage != CRYSTALKV_STAGE_THINK && stage != CRYSTALKV_STAGE_ANSWER) return fail(h, CRYSTALKV_EINVAL, "bad stage");
   if (stage == CRYSTALKV_STAGE_THINK && h->answer_steps > 0)
     return fail(h, CRYSTALKV_ESTATE, "answer tokens were appended; the think stage cannot resume");
+  if (stage != h->stage) CK(h, cudaStreamSynchronize(h->side));   // no LRFU kernel is left behind the switch
   h->stage = stage;
   return CRYSTALKV_OK;
 }
@@ -341,19 +379,24 @@ int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v, c
   if (h->t_layer[layer] >= 0) return fail(h, CRYSTALKV_ESTATE, "layer already prefilled");
   CK(h, cudaSetDevice(c.device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rc = join_side(h, s);   // the insertion pops slots; no LRFU kernel may push or pop meanwhile
+  if (rc) return rc;
   prefill_insert_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer,
                                             static_cast<const __nv_bfloat16*>(k),
                                             static_cast<const __nv_bfloat16*>(v), P);
   CK(h, cudaGetLastError());
   if (evict) {
     // one Algorithm 1 pass with Q^last at t = P-1: seeds CRF/tau, evicts down to the budget
-    DecodeParams p = make_params(h, layer);
+    DecodeParams p = make_params(h, layer, 0);
     p.q = static_cast<const __nv_bfloat16*>(q_last);
     p.k_new = p.v_new = nullptr;
     p.out = h->dummy_out;
     p.t = P - 1;
     p.append = 0; p.track = 1; p.release = 1;
-    CK(h, launch_dispatch(h->G, p, h->grid, h->smem, s));
+    rc = launch_step(h, p, layer, s);
+    if (rc) return rc;
+    rc = join_side(h, s);
+    if (rc) return rc;
     h->par[layer] ^= 1;
   }
   h->t_layer[layer] = P - 1;
@@ -375,14 +418,15 @@ int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* 
     const int used = h->answer_steps / c.n_layers;
     if (used >= c.max_answer_tokens) return fail(h, CRYSTALKV_ESTATE, "max_answer_tokens reached");
   }
-  DecodeParams p = make_params(h, layer);
+  DecodeParams p = make_params(h, layer, 0);
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.k_new = static_cast<const __nv_bfloat16*>(k_new);
   p.v_new = static_cast<const __nv_bfloat16*>(v_new);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.t = t;
   p.append = 1; p.track = track ? 1 : 0; p.release = 0;
-  CK(h, launch_dispatch(h->G, p, h->grid, h->smem, static_cast<cudaStream_t>(stream)));
+  rc = launch_step(h, p, layer, static_cast<cudaStream_t>(stream));
+  if (rc) return rc;
   h->par[layer] ^= 1;
   h->t_layer[layer] = t;
   if (!track && c.mode == CRYSTALKV_MODE_EVICT) h->answer_steps++;
@@ -416,6 +460,7 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   for (int l = 1; l < c.n_layers; ++l)
     if (h->t_layer[l] != t_last || h->par[l] != par) return fail(h, CRYSTALKV_ESTATE, "layers are at different time steps");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   int* n_cur = h->st.nbuf[par];
   crf_sum_kernel<<<h->units, NT, 0, s>>>(h->st, n_cur, t_last, h->Asum);
   CK(h, cudaGetLastError());
@@ -425,7 +470,7 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   const long long B_total = (long long)c.budget_per_head * N;
   alg2_kernel<<<c.batch, NT, sm, s>>>(h->Asum, h->st.budget, c.n_layers, c.n_kv_heads, B_total, c.min_budget, c.max_budget);
   CK(h, cudaGetLastError());
-  const Scratch& sc = h->sc[h->sc_idx];
+  const Scratch& sc = h->sc[0];
   for (int l = 0; l < c.n_layers; ++l) {
     shrink_kernel<<<h->U, NT, 0, s>>>(h->st, n_cur, l, t_last, reinterpret_cast<int*>(sc.pbar), sc.cap_s);
     CK(h, cudaGetLastError());
@@ -440,11 +485,12 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
   if (c.mode != CRYSTALKV_MODE_EVICT) return fail(h, CRYSTALKV_ESTATE, "set_budget in FullKV mode");
   if (budget < 1 || budget > c.max_budget) return fail(h, CRYSTALKV_EINVAL, "budget outside [1, max_budget]");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
   CK(h, cudaMemcpyAsync(h->st.budget + uid, &budget, sizeof(int), cudaMemcpyHostToDevice, s));
   CK(h, cudaStreamSynchronize(s));
   if (h->t_layer[layer] >= 0) {
-    const Scratch& sc = h->sc[h->sc_idx];
+    const Scratch& sc = h->sc[0];
     shrink_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer, h->t_layer[layer],
                                       reinterpret_cast<int*>(sc.pbar), sc.cap_s);
     CK(h, cudaGetLastError());
@@ -455,6 +501,7 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
 int crystalkv_get_budgets(crystalkv_t* h, int32_t* out_host, void* stream) {
   if (!h || !out_host) return fail(h, CRYSTALKV_EINVAL, "null argument");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   CK(h, cudaMemcpyAsync(out_host, h->st.budget, (size_t)h->units * sizeof(int), cudaMemcpyDeviceToHost, s));
   CK(h, cudaStreamSynchronize(s));
   return CRYSTALKV_OK;
@@ -467,6 +514,7 @@ int crystalkv_export_state(crystalkv_t* h, int layer, int seq, int kv_head, int3
   if (!host_buf || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
   int n = 0;
   CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -500,6 +548,7 @@ int crystalkv_get_retained(crystalkv_t* h, int layer, int seq, int kv_head, int3
   if (!pos_out_host || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
   int n = 0;
   CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -519,6 +568,7 @@ int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head, cons
   if (!host_buf || n_rec < 0) return fail(h, CRYSTALKV_EINVAL, "null argument");
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
   int n = 0;
   CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -549,6 +599,7 @@ int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t*
                            uint64_t* evictions, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   unsigned long long v[4];
   CK(h, cudaMemcpyAsync(v, h->st.counters, sizeof(v), cudaMemcpyDeviceToHost, s));
   CK(h, cudaStreamSynchronize(s));
@@ -565,6 +616,7 @@ int crystalkv_validate(crystalkv_t* h, void* stream) {
   for (int l = 0; l < c.n_layers; ++l)
     if (h->t_layer[l] < 0) return fail(h, CRYSTALKV_ESTATE, "validate before every layer is prefilled");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   const long long total = (long long)c.batch * h->slots_per_seq;
   int* seen = nullptr;
   CK(h, cudaMalloc(&seen, (size_t)(total + 2) * sizeof(int)));
@@ -587,9 +639,16 @@ int crystalkv_validate(crystalkv_t* h, void* stream) {
   return CRYSTALKV_OK;
 }
 
+int crystalkv_join(crystalkv_t* h, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  return join_side(h, static_cast<cudaStream_t>(stream));
+}
+
 int crystalkv_check(crystalkv_t* h, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
   int w = 0;
   CK(h, cudaMemcpyAsync(&w, h->st.errword, sizeof(int), cudaMemcpyDeviceToHost, s));
   CK(h, cudaStreamSynchronize(s));
