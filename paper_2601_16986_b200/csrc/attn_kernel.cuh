@@ -38,6 +38,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start while the kernel before it in the stream still runs; pdl_wait() returns once that
+// kernel has completed and its writes are visible, pdl_launch() lets the kernel after this
+// one start.  Both are no-ops for a launch without the attribute.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 // Byte offset of 16-byte chunk `c` of row `r` inside a 16 x 256 B tile; the XOR spreads the
 // eight rows an ldmatrix touches over all banks.
 __device__ __forceinline__ uint32_t tile_off(int r, int c) { return (uint32_t)(r * ROW_BYTES + ((c ^ (r & 7)) << 4)); }
@@ -45,14 +52,19 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) { return (uint32_t)(r
 // One streamed group as the issuing side sees it.
 struct GroupDesc {
   int u;       // head index within the launch (seq * H + kv head)
-  int base;    // list position of the group's first entry
   int valid;   // entries in the group (1..16)
+  int has_new; // the group's last entry is the arriving token
   int slot;    // lane e < valid: pool slot of entry base + e
+  const unsigned char* pool;   // the sequence's pool, advanced to this lane's 16-byte chunk
 };
 
+constexpr float LAZY = 8.0f;   // the running maximum (log2 domain) may trail the true one by this much
+
 __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
-  extern __shared__ __align__(128) unsigned char smem[];
+  extern __shared__ __align__(1024) unsigned char smem[];
   const State& st = p.st;
+  // Without `early` the kernel before this one may still be writing the lists this one reads.
+  if (!p.early) pdl_wait();
   const int U = st.batch * st.H;
   int* off = reinterpret_cast<int*>(smem + RING_BYTES);   // U + 1 group prefix sums
   int* nin = off + (U + 1);                               // U entry counts before the step
@@ -81,26 +93,29 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
     if (tid == 0) off[U] = run;
     __syncthreads();
   }
-  const long long Gtot = off[U];
+  const unsigned Gtot = (unsigned)off[U];
   if (Gtot == 0) return;
-  const int nWarps = gridDim.x * NW;
-  const int nActive = (int)min((long long)nWarps, max(1ll, Gtot / GMIN));
-  const int me = w * gridDim.x + blockIdx.x;   // ranks interleave over the CTAs so small launches use every SM
-  if (me >= nActive) return;
-  const int lo = (int)((long long)me * Gtot / nActive), hi = (int)((long long)(me + 1) * Gtot / nActive);
-  if (hi <= lo) return;
-  auto rank_of = [&](int x) {   // rank of the warp whose range holds group x
-    int c = (int)((long long)x * nActive / Gtot);
-    while ((int)((long long)(c + 1) * Gtot / nActive) <= x) ++c;
-    while ((int)((long long)c * Gtot / nActive) > x) --c;
-    return c;
-  };
+  const unsigned nWarps = gridDim.x * NW;
+  const unsigned per = max((unsigned)GMIN, (Gtot + nWarps - 1) / nWarps);   // groups per working warp
+  const unsigned me = w * gridDim.x + blockIdx.x;   // ranks interleave over the CTAs so small launches use every SM
+  if ((unsigned long long)me * per >= Gtot) return;
+  const int lo = (int)(me * per), hi = (int)min(me * per + per, Gtot);
 
-  unsigned char* ring = smem + (size_t)w * STAGES * STAGE_BYTES;
-  const uint32_t ring_u32 = smem_u32(ring);
+  const uint32_t ring_u32 = smem_u32(smem) + w * (STAGES * STAGE_BYTES);
   const int gid = lane >> 2, tig = lane & 3;
   const int mi = lane >> 3, r8 = lane & 7;
   const int chunk = lane & 15;
+  const uint32_t half_off = lane < 16 ? 0u : (uint32_t)(GRP * ROW_BYTES);
+  // cp.async destination of this lane's chunk in row e of a stage: xoff[e & 7] + e * 256
+  uint32_t xoff[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) xoff[j] = half_off + (uint32_t)((chunk ^ j) << 4);
+  // ldmatrix row addresses: K tile of k-step ks at (stage + kb) ^ (ks << 5), V tile of channel
+  // tile mt at (stage + vb) ^ (mt << 5); stages are 256-byte aligned so the XOR is carry free
+  const uint32_t kb = (uint32_t)(((mi & 1) * 8 + r8) * ROW_BYTES + (((mi >> 1) ^ r8) << 4));
+  const uint32_t vb = (uint32_t)(GRP * ROW_BYTES + ((mi >> 1) * 8 + r8) * ROW_BYTES + (((mi & 1) ^ r8) << 4));
+  const unsigned char* newrow_lane =
+      reinterpret_cast<const unsigned char*>(lane < 16 ? p.k_new : p.v_new) + chunk * 16;
 
   // first head whose group range holds `lo`
   int u_first = 0;
@@ -113,52 +128,76 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
     u_first = a;
   }
 
-  // ---- issuing side
-  int iu = u_first;
+  // ---- issuing side: registers of the head whose groups are being requested
+  int iu = u_first, i_seq = u_first / st.H, i_head = u_first % st.H;
+  int i_off, i_end, i_ntot;
+  const int* i_list;
+  const unsigned char* i_pool;
+  auto issue_unit = [&]() {
+    i_off = off[iu];
+    i_end = off[iu + 1];
+    i_ntot = nin[iu] + p.append;
+    const int uid = (i_seq * st.L + p.layer) * st.H + i_head;
+    i_list = st.list_slot + (size_t)uid * st.cap;
+    i_pool = st.pool + (size_t)i_seq * st.slots_per_seq * SLOT_BYTES + lane * 16;
+  };
+  issue_unit();
   auto prep = [&](int idx) {
+    if (idx >= i_end) {
+      do {
+        ++iu;
+        if (++i_head == st.H) { i_head = 0; ++i_seq; }
+      } while (off[iu + 1] <= idx);
+      issue_unit();
+    }
     GroupDesc d;
-    while (off[iu + 1] <= idx) ++iu;
+    const int base = (idx - i_off) * GRP;
     d.u = iu;
-    d.base = (idx - off[iu]) * GRP;
-    d.valid = min(GRP, nin[iu] + p.append - d.base);
-    const int uid = ((iu / st.H) * st.L + p.layer) * st.H + (iu % st.H);
-    d.slot = (lane < d.valid) ? st.list_slot[(size_t)uid * st.cap + d.base + lane] : 0;
+    d.valid = min(GRP, i_ntot - base);
+    d.has_new = p.append && (base + d.valid == i_ntot);
+    d.slot = (lane < d.valid) ? i_list[base + lane] : 0;
+    d.pool = i_pool;
     return d;
   };
-  auto fire = [&](const GroupDesc& d, int stage) {
-    const int seq = d.u / st.H, head = d.u % st.H;
-    const unsigned char* poolseq = st.pool + (size_t)seq * st.slots_per_seq * SLOT_BYTES;
-    const int n_old = nin[d.u];
-    const int e_new = (p.append && n_old >= d.base && n_old < d.base + GRP) ? n_old - d.base : -1;
-    const uint32_t dst0 = ring_u32 + stage * STAGE_BYTES + (lane < 16 ? 0 : GRP * ROW_BYTES);
+  auto fire = [&](const GroupDesc& d, uint32_t stage) {
+    if (d.valid == GRP && !d.has_new) {
 #pragma unroll
-    for (int e = 0; e < GRP; ++e) {
-      const int s = __shfl_sync(0xffffffffu, d.slot, e);
-      const uint32_t dst = dst0 + tile_off(e, chunk);
-      if (e < d.valid) {
-        const unsigned char* src = poolseq + (size_t)s * SLOT_BYTES + lane * 16;
-        if (e == e_new)   // the arriving token comes from the call's inputs
-          src = reinterpret_cast<const unsigned char*>((lane < 16 ? p.k_new : p.v_new) + ((size_t)seq * st.H + head) * HD) + chunk * 16;
-        cp_async16(dst, src);
-      } else {
-        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};\n" ::"r"(dst), "r"(0) : "memory");
+      for (int e = 0; e < GRP; ++e) {
+        const unsigned s = (unsigned)__shfl_sync(0xffffffffu, d.slot, e);
+        cp_async16(stage + xoff[e & 7] + e * ROW_BYTES, d.pool + (size_t)s * SLOT_BYTES);
+      }
+    } else {
+      const int nv = d.valid - d.has_new;   // entries that come from the pool
+#pragma unroll
+      for (int e = 0; e < GRP; ++e) {
+        const unsigned s = (unsigned)__shfl_sync(0xffffffffu, d.slot, e);
+        const uint32_t dst = stage + xoff[e & 7] + e * ROW_BYTES;
+        if (e < nv) {
+          cp_async16(dst, d.pool + (size_t)s * SLOT_BYTES);
+        } else if (e >= d.valid) {
+          asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};\n" ::"r"(dst), "r"(0) : "memory");
+        }
+      }
+      if (d.has_new) {   // the arriving token comes from the call's inputs
+        pdl_wait();
+        const int e = d.valid - 1;
+        cp_async16(stage + half_off + tile_off(e, chunk), newrow_lane + (size_t)d.u * ROW_BYTES);
       }
     }
   };
 
   // ---- computing side: state of the head being accumulated
-  int cu = -1;
+  int cu = -1, c_seq = 0, c_head = 0, c_off = 0, c_end = 0, c_nold = 0;
+  float* c_logit = nullptr;
   uint32_t qb[8][2];
   float o[8][4];
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
   auto publish = [&]() {
     const int u = cu;
-    const int seq = u / st.H, head = u % st.H;
-    const int uid = (seq * st.L + p.layer) * st.H + head;
-    const int g0 = off[u], g1 = off[u + 1];
-    const int r_first = rank_of(g0), r_last = rank_of(g1 - 1);
-    const int piece = me - r_first, npieces = r_last - r_first + 1;
+    const int uid = (c_seq * st.L + p.layer) * st.H + c_head;
+    const unsigned r_first = (unsigned)c_off / per, r_last = (unsigned)(c_end - 1) / per;
+    const int piece = (int)(me - r_first), npieces = (int)(r_last - r_first + 1);
     float* part = p.sc.partials + ((size_t)u * p.sc.pmax + piece) * PS;
     // l over the keys of all lanes that hold the same heads
     float ls0 = l0, ls1 = l1;
@@ -168,15 +207,15 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
       ls1 += __shfl_xor_sync(0xffffffffu, ls1, x);
     }
     if (gid == 0) {
-      part[2 * tig] = m0; part[2 * tig + 1] = m1;
-      part[8 + 2 * tig] = ls0; part[8 + 2 * tig + 1] = ls1;
+      *reinterpret_cast<float2*>(part + 2 * tig) = make_float2(m0, m1);
+      *reinterpret_cast<float2*>(part + 8 + 2 * tig) = make_float2(ls0, ls1);
     }
     const int h0 = 2 * tig, h1 = 2 * tig + 1;
+    float* po = part + 16 + gid;
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
-      const int d0 = 16 * mt + gid;
-      if (h0 < G) { part[16 + h0 * HD + d0] = o[mt][0]; part[16 + h0 * HD + d0 + 8] = o[mt][2]; }
-      if (h1 < G) { part[16 + h1 * HD + d0] = o[mt][1]; part[16 + h1 * HD + d0 + 8] = o[mt][3]; }
+      if (h0 < G) { po[h0 * HD + 16 * mt] = o[mt][0]; po[h0 * HD + 16 * mt + 8] = o[mt][2]; }
+      if (h1 < G) { po[h1 * HD + 16 * mt] = o[mt][1]; po[h1 * HD + 16 * mt + 8] = o[mt][3]; }
     }
     __threadfence();
     __syncwarp();
@@ -189,41 +228,76 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) return;
     __threadfence();
-    // ---- merge: out = sum_p O_p 2^(m_p - m) / sum_p l_p 2^(m_p - m), lane = 4 output channels
+    // ---- merge: out = sum_p O_p 2^(m_p - m) / sum_p l_p 2^(m_p - m).  Loads that do not depend
+    // on one another are issued together: first every piece's (m, l) header, then the O rows.
     const float* pbase = p.sc.partials + (size_t)u * p.sc.pmax * PS;
     const int Hq = st.H * G;
-    for (int g = 0; g < G; ++g) {
-      float mm = -INFINITY;
-      for (int pc = 0; pc < npieces; ++pc) mm = fmaxf(mm, __ldcg(pbase + (size_t)pc * PS + g));
-      float L = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int pc = 0; pc < npieces; ++pc) {
-        const float* pp = pbase + (size_t)pc * PS;
-        const float sc = ex2(__ldcg(pp + g) - mm);
-        L = fmaf(__ldcg(pp + 8 + g), sc, L);
-        const float4 ov = __ldcg(reinterpret_cast<const float4*>(pp + 16 + g * HD) + lane);
-        acc.x = fmaf(ov.x, sc, acc.x); acc.y = fmaf(ov.y, sc, acc.y);
-        acc.z = fmaf(ov.z, sc, acc.z); acc.w = fmaf(ov.w, sc, acc.w);
-      }
-      const float inv = 1.0f / L;
-      uint2 pk;
-      pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-      pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-      *reinterpret_cast<uint2*>(p.out + ((size_t)seq * Hq + head * G + g) * HD + lane * 4) = pk;
-      if (lane == 0 && p.track) p.sc.mfin[u * QH + g] = mm;
+    const int hh = lane & 7, pl = lane >> 3;   // header phase: lane = (piece mod 4, head)
+    float mm = -INFINITY;
+    for (int pc = pl; pc < npieces; pc += 4) mm = fmaxf(mm, __ldcg(pbase + (size_t)pc * PS + hh));
+    mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, 8));
+    mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, 16));
+    float Ls = 0.f;
+    for (int pc = pl; pc < npieces; pc += 4)
+      Ls = fmaf(__ldcg(pbase + (size_t)pc * PS + 8 + hh), ex2(__ldcg(pbase + (size_t)pc * PS + hh) - mm), Ls);
+    Ls += __shfl_xor_sync(0xffffffffu, Ls, 8);
+    Ls += __shfl_xor_sync(0xffffffffu, Ls, 16);
+    if (lane < G && p.track) {   // reference point and normaliser of the step's softmax, for the LRFU kernel
+      p.sc.mfin[u * (2 * QH) + lane] = mm;
+      p.sc.mfin[u * (2 * QH) + QH + lane] = Ls;
     }
+    float mg[QH], inv[QH];
+#pragma unroll
+    for (int g = 0; g < QH; ++g) {
+      mg[g] = __shfl_sync(0xffffffffu, mm, g);
+      inv[g] = 1.0f / __shfl_sync(0xffffffffu, Ls, g);
+    }
+    float4 acc[QH];   // lane = 4 output channels of every head
+#pragma unroll
+    for (int g = 0; g < QH; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int pc = 0; pc < npieces; ++pc) {
+      const float* pp = pbase + (size_t)pc * PS;
+#pragma unroll
+      for (int g = 0; g < QH; ++g) {
+        if (g < G) {
+          const float sc = ex2(__ldcg(pp + g) - mg[g]);
+          const float4 ov = __ldcg(reinterpret_cast<const float4*>(pp + 16 + g * HD) + lane);
+          acc[g].x = fmaf(ov.x, sc, acc[g].x); acc[g].y = fmaf(ov.y, sc, acc[g].y);
+          acc[g].z = fmaf(ov.z, sc, acc[g].z); acc[g].w = fmaf(ov.w, sc, acc[g].w);
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < QH; ++g) {
+      if (g < G) {
+        uint2 pk;
+        pk.x = pack_bf16(acc[g].x * inv[g], acc[g].y * inv[g]);
+        pk.y = pack_bf16(acc[g].z * inv[g], acc[g].w * inv[g]);
+        *reinterpret_cast<uint2*>(p.out + ((size_t)(u * G + g)) * HD + lane * 4) = pk;
+      }
+    }
+    (void)Hq;
     if (lane == 0) {
-      const int n_tot = nin[u] + p.append;
+      const int n_tot = c_nold + p.append;
       atomicAdd(&st.counters[0], (unsigned long long)n_tot);
-      if (!p.track) keep_and_refill(st, p.n_out, uid, seq, n_tot, p.append != 0);
+      if (!p.track) keep_and_refill(st, p.n_out, uid, c_seq, n_tot, p.append != 0);
     }
   };
 
   auto enter = [&](int idx) {   // start accumulating the head that holds group idx
-    cu = (cu < 0) ? u_first : cu + 1;
-    while (off[cu + 1] <= idx) ++cu;
-    const int seq = cu / st.H, head = cu % st.H;
-    const uint32_t* q32 = reinterpret_cast<const uint32_t*>(p.q + ((size_t)seq * st.H * G + head * G + gid) * HD);
+    if (cu < 0) {
+      cu = u_first; c_seq = u_first / st.H; c_head = u_first % st.H;
+    } else {
+      do {
+        ++cu;
+        if (++c_head == st.H) { c_head = 0; ++c_seq; }
+      } while (off[cu + 1] <= idx);
+    }
+    c_off = off[cu];
+    c_end = off[cu + 1];
+    c_nold = nin[cu];
+    c_logit = p.sc.logits + (size_t)cu * p.sc.cap_s * QH + gid * QH + 2 * tig;
+    const uint32_t* q32 = reinterpret_cast<const uint32_t*>(p.q + ((size_t)cu * G + gid) * HD);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       qb[ks][0] = (gid < G) ? q32[ks * 8 + tig] : 0u;
@@ -234,45 +308,42 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
     m0 = -INFINITY; m1 = -INFINITY; l0 = 0.f; l1 = 0.f;
   };
 
-  auto compute = [&](int idx, int stage) {
-    const int u = cu;
-    const int base = (idx - off[u]) * GRP;
-    const int n_old = nin[u], n_tot = n_old + p.append;
+  auto compute = [&](int idx, uint32_t stage) {
+    const int base = (idx - c_off) * GRP;
+    const int n_tot = c_nold + p.append;
     const int valid = min(GRP, n_tot - base);
-    const uint32_t sK = ring_u32 + stage * STAGE_BYTES, sV = sK + GRP * ROW_BYTES;
-    if (p.append && n_old >= base && n_old < base + GRP) {
+    if (p.append && base + valid == n_tot) {
       // the arriving token: its rows go from the stage into the head's spare slot
-      const int seq = u / st.H;
-      const int uid = (seq * st.L + p.layer) * st.H + (u % st.H);
+      const int uid = (c_seq * st.L + p.layer) * st.H + c_head;
       const size_t mb = (size_t)uid * st.cap;
-      const int e = n_old - base;
-      const int slot = st.list_slot[mb + n_old];
+      const int e = valid - 1;
+      const int slot = st.list_slot[mb + c_nold];
       uint4 val;
-      const uint32_t src = (lane < 16 ? sK : sV) + tile_off(e, chunk);
+      const uint32_t src = stage + half_off + tile_off(e, chunk);
       asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];\n" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(src));
-      *reinterpret_cast<uint4*>(st.pool + ((size_t)seq * st.slots_per_seq + slot) * SLOT_BYTES + lane * 16) = val;
+      *reinterpret_cast<uint4*>(st.pool + ((size_t)c_seq * st.slots_per_seq + slot) * SLOT_BYTES + lane * 16) = val;
       if (lane == 0) {
-        st.meta_pos[mb + n_old] = p.t;
-        st.meta_tau[mb + n_old] = p.t;
-        st.meta_crf[mb + n_old] = 0.0f;
+        st.meta_pos[mb + c_nold] = p.t;
+        st.meta_tau[mb + c_nold] = p.t;
+        st.meta_crf[mb + c_nold] = 0.0f;
       }
     }
     // ---- S[key][head] = K Q^T over the 8 k-steps of 16 channels
     float s[4] = {0.f, 0.f, 0.f, 0.f};
     {
-      const int krow = (mi & 1) * 8 + r8;
+      const uint32_t ka = stage + kb;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         uint32_t a[4];
-        ldsm_x4(a, sK + tile_off(krow, 2 * ks + (mi >> 1)));
+        ldsm_x4(a, ka ^ (uint32_t)(ks << 5));
         mma_bf16(s, a, qb[ks][0], qb[ks][1]);
       }
     }
     const bool v0 = gid < valid, v1 = gid + 8 < valid;
     if (p.track) {
-      float* lrow = p.sc.logits + ((size_t)u * p.sc.cap_s + base) * QH + 2 * tig;
-      if (v0) *reinterpret_cast<float2*>(lrow + (size_t)gid * QH) = make_float2(__fmul_rn(s[0], p.scale), __fmul_rn(s[1], p.scale));
-      if (v1) *reinterpret_cast<float2*>(lrow + (size_t)(gid + 8) * QH) = make_float2(__fmul_rn(s[2], p.scale), __fmul_rn(s[3], p.scale));
+      float* lrow = c_logit + (size_t)base * QH;
+      if (v0) *reinterpret_cast<float2*>(lrow) = make_float2(__fmul_rn(s[0], p.scale), __fmul_rn(s[1], p.scale));
+      if (v1) *reinterpret_cast<float2*>(lrow + 8 * QH) = make_float2(__fmul_rn(s[2], p.scale), __fmul_rn(s[3], p.scale));
     }
     // ---- online softmax, this lane's two heads (2 tig, 2 tig + 1) over its two keys
     const float t0 = v0 ? s[0] * p.scale_log2 : -INFINITY, t1 = v0 ? s[1] * p.scale_log2 : -INFINITY;
@@ -283,8 +354,10 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
       c0 = fmaxf(c0, __shfl_xor_sync(0xffffffffu, c0, x));
       c1 = fmaxf(c1, __shfl_xor_sync(0xffffffffu, c1, x));
     }
-    const float n0 = fmaxf(m0, c0), n1 = fmaxf(m1, c1);
-    if (__any_sync(0xffffffffu, n0 > m0 || n1 > m1)) {
+    // the reference point only moves when a maximum has grown by more than LAZY, so most groups
+    // skip the rescale; weights stay below 2^LAZY
+    if (__any_sync(0xffffffffu, c0 > m0 + LAZY || c1 > m1 + LAZY)) {
+      const float n0 = fmaxf(m0, c0), n1 = fmaxf(m1, c1);
       const float r0 = ex2(m0 - n0), r1 = ex2(m1 - n1);
       l0 *= r0; l1 *= r1;
 #pragma unroll
@@ -294,50 +367,63 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
     const float p0 = ex2(t0 - m0), p1 = ex2(t1 - m1), p2 = ex2(t2 - m0), p3 = ex2(t3 - m1);
     l0 += p0 + p2;
     l1 += p1 + p3;
-    // P^T as the B operand: transpose the two 8 x 8 (key x head) blocks across the warp
-    const uint32_t b0 = movm_t(pack_bf16(p0, p1)), b1 = movm_t(pack_bf16(p2, p3));
+    // P^T as the B operand: transpose the two 8 x 8 (key x head) blocks across the warp.  The
+    // weights go in as a bf16 head plus a bf16 remainder, which keeps 16 bits of each.
+    const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
+    const uint32_t b0 = movm_t(*reinterpret_cast<const uint32_t*>(&h01)), b1 = movm_t(*reinterpret_cast<const uint32_t*>(&h23));
+    const uint32_t r0 = movm_t(pack_bf16(p0 - __low2float(h01), p1 - __high2float(h01)));
+    const uint32_t r1 = movm_t(pack_bf16(p2 - __low2float(h23), p3 - __high2float(h23)));
     // ---- O^T[channel][head] += V^T P^T, 8 tiles of 16 channels
     {
-      const int vrow = (mi >> 1) * 8 + r8;
+      const uint32_t va = stage + vb;
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) {
         uint32_t a[4];
-        ldsm_x4_t(a, sV + tile_off(vrow, 2 * mt + (mi & 1)));
+        ldsm_x4_t(a, va ^ (uint32_t)(mt << 5));
         mma_bf16(o[mt], a, b0, b1);
+        mma_bf16(o[mt], a, r0, r1);
       }
     }
   };
 
-  // ---- the pipeline: groups lo .. hi-1 flow through the ring, STAGES-1 of them in flight
-  GroupDesc nd = prep(lo);
+  // ---- the pipeline: groups lo .. hi-1 flow through the ring, STAGES-1 of them in flight; the
+  // slot ids of a group are requested two fires before they are needed
+  GroupDesc nd0 = prep(lo), nd1 = nd0;
+  if (lo + 1 < hi) nd1 = prep(lo + 1);
   int next = lo;   // next group to fire
-#pragma unroll 1
-  for (int s = 0; s < STAGES - 1; ++s) {
+  uint32_t fs = ring_u32;   // stage the next fire fills
+  auto fire_next = [&]() {
     if (next < hi) {
-      const GroupDesc d = nd;
+      const GroupDesc d = nd0;
+      nd0 = nd1;
+      if (next + 2 < hi) nd1 = prep(next + 2);
       ++next;
-      if (next < hi) nd = prep(next);
-      fire(d, s);
+      fire(d, fs);
     }
     cp_commit();
-  }
+    fs += STAGE_BYTES;
+  };
+  const uint32_t ring_end = ring_u32 + STAGES * STAGE_BYTES;
+#pragma unroll 1
+  for (int s = 0; s < STAGES - 1; ++s) fire_next();
+  // everything above reads only the cache and its lists; the call's inputs (q, the arriving
+  // row is fetched by the cp.async of a head's last group) may come from the kernel before
+  pdl_wait();
+  pdl_launch();
+  uint32_t cs = ring_u32;   // stage the next compute reads
 #pragma unroll 1
   for (int ci = lo; ci < hi; ++ci) {
-    const int k = ci - lo;
-    if (next < hi) {
-      const GroupDesc d = nd;
-      ++next;
-      if (next < hi) nd = prep(next);
-      fire(d, (k + STAGES - 1) % STAGES);
-    }
-    cp_commit();
+    fire_next();
+    if (fs == ring_end) fs = ring_u32;
     cp_wait<STAGES - 1>();
     __syncwarp();
-    if (cu < 0 || ci >= off[cu + 1]) {
+    if (ci >= c_end) {
       if (cu >= 0) publish();
       enter(ci);
     }
-    compute(ci, k % STAGES);
+    compute(ci, cs);
+    cs += STAGE_BYTES;
+    if (cs == ring_end) cs = ring_u32;
     __syncwarp();   // the stage is free for the fire of the next iteration
   }
   publish();

@@ -50,7 +50,7 @@ struct Scratch {
   float* logits;     // [U][cap_s][QH] scaled logits of the step, one 32-byte row per entry
   float* pbar;       // [U][cap_s] group-mean probabilities (reused as int scratch)
   float* partials;   // [U][pmax][16 + G*128] split-K partial: m[8], l[8], O[G][128]
-  float* mfin;       // [U][QH] merged running maximum (log2 domain) per query head
+  float* mfin;       // [U][2][QH] per query head: merged reference point (log2 domain), then normaliser
   int* ticket;       // [U]
   int cap_s, pmax;
 };
@@ -70,6 +70,8 @@ struct DecodeParams {
   int append;     // 1: decode (a new entry arrives); 0: scoring pass over the prompt
   int track;      // 1: Algorithm 1 runs (hits, CRF, eviction) in the LRFU kernel that follows
   int release;    // 1: freed slots beyond one spare go back to the free list (no pops in this launch)
+  int early;      // 1: the lists and rows of this layer are final, so the attention kernel may read them
+                  //    before the kernel ahead of it in the stream has completed
   float scale;    // logit scale
   float scale_log2;
   float top_p;

@@ -38,6 +38,7 @@ struct crystalkv {
   cudaEvent_t evA = nullptr, evF[EV_RING] = {};
   long long kF = 0, joined = -1;
   std::vector<long long> lastF;    // per layer: number of its latest LRFU launch, -1 = none
+  int prev_layer = -1;             // layer of the launch pair issued last, -1 after any other call
   int stage = CRYSTALKV_STAGE_THINK;
   int answer_steps = 0;
   long long* Asum = nullptr;
@@ -100,6 +101,15 @@ __global__ void fill_int_kernel(int* p, long long n, int v) {
 
 template <int G>
 cudaError_t launch_lrfu(const DecodeParams& p, int grid, cudaStream_t s) {
+  // the same shared-memory carve-out as the attention kernel, so that CTAs of both can be
+  // resident on one SM at the same time
+  static bool prepared = false;
+  if (!prepared) {
+    cudaError_t e = cudaFuncSetAttribute(lrfu_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         (int)cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    prepared = true;
+  }
   lrfu_kernel<G><<<grid, NT, 0, s>>>(p);
   return cudaGetLastError();
 }
@@ -170,6 +180,7 @@ DecodeParams make_params(crystalkv_t* h, int layer, int set) {
 
 // Makes `s` wait for every LRFU kernel launched so far.
 int join_side(crystalkv_t* h, cudaStream_t s) {
+  h->prev_layer = -1;
   if (h->kF > 0) CK(h, cudaStreamWaitEvent(s, h->evF[(h->kF - 1) % crystalkv::EV_RING], 0));
   h->joined = h->kF - 1;
   return CRYSTALKV_OK;
@@ -189,8 +200,25 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
     }
     p.sc = h->sc[k % NSETS];
   }
-  attn_kernel<<<h->grid, NT, h->smem, s>>>(p);
-  CK(h, cudaGetLastError());
+  // The attention kernel may start while the kernel ahead of it still runs: it first fills its
+  // pipeline from the cache and waits for that kernel before it touches the call's inputs.
+  // That is only sound if the kernel ahead cannot be writing this layer's lists, which holds
+  // when it is the attention kernel of another layer.
+  p.early = (h->prev_layer >= 0 && h->prev_layer != layer) ? 1 : 0;
+  {
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(h->grid);
+    lc.blockDim = dim3(NT);
+    lc.dynamicSmemBytes = h->smem;
+    lc.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    CK(h, cudaLaunchKernelEx(&lc, attn_kernel, p));
+  }
+  h->prev_layer = layer;
   if (track) {
     CK(h, cudaEventRecord(h->evA, s));
     CK(h, cudaStreamWaitEvent(h->side, h->evA, 0));
@@ -319,7 +347,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     DA(&sc.logits, (size_t)h->U * sc.cap_s * QH);
     DA(&sc.pbar, (size_t)h->U * sc.cap_s);
     DA(&sc.partials, (size_t)h->U * sc.pmax * (16 + h->G * HD));
-    DA(&sc.mfin, (size_t)h->U * QH);
+    DA(&sc.mfin, (size_t)h->U * 2 * QH);
     DA(&sc.ticket, h->U);
     CKC(cudaMemset(sc.ticket, 0, (size_t)h->U * sizeof(int)));
   }
@@ -356,6 +384,7 @@ int crystalkv_set_stage(crystalkv_t* h, int stage) {
   if (stage == CRYSTALKV_STAGE_THINK && h->answer_steps > 0)
     return fail(h, CRYSTALKV_ESTATE, "answer tokens were appended; the think stage cannot resume");
   if (stage != h->stage) CK(h, cudaStreamSynchronize(h->side));   // no LRFU kernel is left behind the switch
+  h->prev_layer = -1;
   h->stage = stage;
   return CRYSTALKV_OK;
 }

@@ -1,13 +1,15 @@
 // Algorithm 1 for the heads of one layer, one CTA per head, from the scaled logits the
 // attention kernel left in the scratch (the cache itself is not read again):
-//   step 1   exact softmax per query head (accurate expf, fixed reduction order), group-mean
-//            probability pbar, hit mask = smallest descending-pbar prefix whose exclusive
-//            mass is below p (equal pbar: ascending position);
+//   step 1   softmax weights per query head from the logits, the attention kernel's merged
+//            reference point and normaliser (accurate expf), group-mean probability pbar,
+//            hit mask = smallest descending-pbar prefix whose exclusive mass is below p
+//            (equal pbar: ascending position);
 //   step 2-3 hits: CRF <- lambda^(t - tau) CRF + 1, tau <- t; misses only get the decayed
 //            CRF_temp, which is not stored;
 //   step 4   the entries lowest under (CRF_temp, tau, position) leave until the head is
 //            within its budget; the freed slot is reused in place.
-// The mass walk uses 2^-40 fixed-point integers so it is exact and order independent.
+// The mass walk uses 2^-40 fixed-point integers so it is exact and order independent; the
+// threshold is relative to the integer total, so a common factor on pbar changes nothing.
 #pragma once
 #include "common.cuh"
 #include "evict.cuh"
@@ -15,126 +17,142 @@
 namespace ckv {
 
 constexpr int HIST_BINS = 2048;
+constexpr float MASS_ONE = 1099511627776.0f;   // 2^40
 
-template <int G>
-__global__ void __launch_bounds__(NT) lrfu_kernel(const DecodeParams p) {
-  __shared__ unsigned long long hist[HIST_BINS];
-  __shared__ float redf[NW * 8];
-  __shared__ unsigned long long redu[NW + 4];
-  __shared__ float s_l[8];
-  __shared__ int s_star;
-  __shared__ int s_eq[NW];
-  __shared__ int s_min[NW * 4];
-  __shared__ int sh_ev[320];
+struct LrfuSmem {
+  unsigned hist_lo[HIST_BINS];   // per-bin mass, low 16 bits of every term
+  unsigned hist_hi[HIST_BINS];   // per-bin mass, the bits above
+  unsigned long long redu[NW + 4];
+  int star;
+  int eq[NW];
+  int amin[NW * 4];
+  int ev[320];
+};
+
+__device__ __forceinline__ unsigned long long mass_of(float pm) { return (unsigned long long)(pm * MASS_ONE); }
+
+// EPT > 0: every thread keeps the pbar of its entries tid, tid + NT, ... (at most EPT) in
+// registers; EPT == 0: they live in the global scratch and any n is allowed.
+template <int G, int EPT>
+__device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n, LrfuSmem& sh) {
+  constexpr int R = EPT > 0 ? EPT : 1;
   const State& st = p.st;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
-  const int uid = (seq * st.L + p.layer) * st.H + head;
   const size_t mb = (size_t)uid * st.cap;
-  const int n = p.n_in[uid] + p.append;
-  if (n <= 0) {
-    if (tid == 0) p.n_out[uid] = 0;
-    return;
-  }
   const float* S = p.sc.logits + (size_t)u * p.sc.cap_s * QH;
   float* pbar = p.sc.pbar + (size_t)u * p.sc.cap_s;
+  const int kmax = EPT > 0 ? (n + NT - 1) / NT : 0;
 
-  // ---- step 1a: normalisers, shifted by the attention kernel's running maximum
-  float mx[G], sm[G];
+  // ---- step 1: pbar_i = mean_g exp(s_gi - m_g) / l_g
+  float mx[G], invl[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
-    mx[g] = p.sc.mfin[u * QH + g] * 0.693147180559945309f;   // log2 domain -> natural log
-    sm[g] = 0.f;
+    mx[g] = p.sc.mfin[u * (2 * QH) + g] * 0.693147180559945309f;   // log2 domain -> natural log
+    invl[g] = 1.0f / (p.sc.mfin[u * (2 * QH) + QH + g] * (float)G);
   }
-  for (int i = tid; i < n; i += NT) {
+  auto pbar_of = [&](int i) {
     const float4 a = *reinterpret_cast<const float4*>(S + (size_t)i * QH);
-    const float4 b = *reinterpret_cast<const float4*>(S + (size_t)i * QH + 4);
-    const float sv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-#pragma unroll
-    for (int g = 0; g < G; ++g) sm[g] += expf(sv[g] - mx[g]);
-  }
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const float v = warp_sum(sm[g]);
-    if (lane == 0) redf[w * 8 + g] = v;
-  }
-  __syncthreads();
-  if (tid < G) {
-    float v = redf[tid];
-    for (int x = 1; x < NW; ++x) v += redf[x * 8 + tid];
-    s_l[tid] = v;
-  }
-  __syncthreads();
-  // ---- step 1b: pbar_i = mean_g p_{g,i}; integer mass w_i = floor(pbar_i * 2^40)
-  float li[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) li[g] = s_l[g];
-  unsigned long long wsum = 0;
-  for (int i = tid; i < n; i += NT) {
-    const float4 a = *reinterpret_cast<const float4*>(S + (size_t)i * QH);
-    const float4 b = *reinterpret_cast<const float4*>(S + (size_t)i * QH + 4);
+    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (G > 4) b = *reinterpret_cast<const float4*>(S + (size_t)i * QH + 4);
     const float sv[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     float pm = 0.f;
 #pragma unroll
-    for (int g = 0; g < G; ++g) pm += __fdiv_rn(expf(sv[g] - mx[g]), li[g]);
-    pm = __fdiv_rn(pm, (float)G);
-    pbar[i] = pm;
-    wsum += (unsigned long long)(pm * 1099511627776.0f);
+    for (int g = 0; g < G; ++g) pm = fmaf(expf(sv[g] - mx[g]), invl[g], pm);
+    return pm;
+  };
+  float pmr[R];
+  unsigned long long wsum = 0;
+  if (EPT > 0) {
+#pragma unroll
+    for (int k = 0; k < R; ++k) {
+      const int i = tid + k * NT;
+      pmr[k] = 0.f;
+      if (k < kmax && i < n) {
+        pmr[k] = pbar_of(i);
+        wsum += mass_of(pmr[k]);
+      }
+    }
+  } else {
+    for (int i = tid; i < n; i += NT) {
+      const float pm = pbar_of(i);
+      pbar[i] = pm;
+      wsum += mass_of(pm);
+    }
   }
   wsum = warp_sum_u64(wsum);
-  if (lane == 0) redu[w] = wsum;
+  if (lane == 0) sh.redu[w] = wsum;
   __syncthreads();
   unsigned long long W = 0;
-  for (int x = 0; x < NW; ++x) W += redu[x];
+  for (int x = 0; x < NW; ++x) W += sh.redu[x];
   // hit  <=>  mass strictly before the entry  <  p * W
   const unsigned long long Pthr = (unsigned long long)ceil((double)p.top_p * (double)W);
+
   // ---- threshold key by MSB-first radix passes over the fp32 bits of pbar (11, 11, 10 bits)
   unsigned long long A = 0;   // mass of keys strictly above the current prefix range
   uint32_t prefix = 0;
   bool found_all = true;
-  const int shifts[3] = {21, 10, 0};
-  const int widths[3] = {11, 11, 10};
   for (int pass = 0; pass < 3; ++pass) {
-    const int sh = shifts[pass], nb = 1 << widths[pass];
+    const int sft = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const int wid = pass == 2 ? 10 : 11;
+    const int nb = 1 << wid;
     __syncthreads();
-    for (int b = tid; b < nb; b += NT) hist[b] = 0ull;
-    if (tid == 0) s_star = -1;
+    for (int b = tid; b < nb; b += NT) { sh.hist_lo[b] = 0u; sh.hist_hi[b] = 0u; }
+    if (tid == 0) sh.star = -1;
     __syncthreads();
-    for (int i = tid; i < n; i += NT) {
-      const float pm = pbar[i];
+    auto add = [&](float pm) {
       const uint32_t key = __float_as_uint(pm);
-      const bool match = (pass == 0) || ((key >> (sh + widths[pass])) == (prefix >> (sh + widths[pass])));
-      if (match) atomicAdd(&hist[(key >> sh) & (nb - 1)], (unsigned long long)(pm * 1099511627776.0f));
+      const bool match = (pass == 0) || ((key >> (sft + wid)) == (prefix >> (sft + wid)));
+      if (match) {
+        const unsigned long long m = mass_of(pm);
+        const int b = (key >> sft) & (nb - 1);
+        atomicAdd(&sh.hist_lo[b], (unsigned)(m & 0xffffu));
+        atomicAdd(&sh.hist_hi[b], (unsigned)(m >> 16));
+      }
+    };
+    if (EPT > 0) {
+#pragma unroll
+      for (int k = 0; k < R; ++k)
+        if (k < kmax && tid + k * NT < n) add(pmr[k]);
+    } else {
+      for (int i = tid; i < n; i += NT) add(pbar[i]);
     }
     __syncthreads();
     // suffix sums from the top bin: thread k owns bins [k*per, (k+1)*per)
     const int per = nb / NT;
+    unsigned long long hb[HIST_BINS / NT];
     unsigned long long loc = 0;
-    for (int b = 0; b < per; ++b) loc += hist[tid * per + b];
+#pragma unroll
+    for (int b = 0; b < HIST_BINS / NT; ++b) {
+      hb[b] = 0;
+      if (b < per) hb[b] = ((unsigned long long)sh.hist_hi[tid * per + b] << 16) + sh.hist_lo[tid * per + b];
+      loc += hb[b];
+    }
     unsigned long long suf = loc;   // inclusive suffix scan across the warp (higher lane = higher bins)
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       unsigned long long x = __shfl_down_sync(0xffffffffu, suf, o);
       if (lane + o < 32) suf += x;
     }
-    if (lane == 0) redu[w] = suf;
+    if (lane == 0) sh.redu[w] = suf;
     __syncthreads();
     unsigned long long above = 0;
-    for (int x = w + 1; x < NW; ++x) above += redu[x];
+    for (int x = w + 1; x < NW; ++x) above += sh.redu[x];
     unsigned long long sab = A + above + (suf - loc);   // mass above this thread's top bin
-    for (int b = per - 1; b >= 0; --b) {
-      const unsigned long long hb = hist[tid * per + b];
-      if (sab < Pthr && Pthr <= sab + hb) {
-        s_star = tid * per + b;
-        redu[NW] = sab;
+#pragma unroll
+    for (int b = HIST_BINS / NT - 1; b >= 0; --b) {
+      if (b < per) {
+        if (sab < Pthr && Pthr <= sab + hb[b]) {
+          sh.star = tid * per + b;
+          sh.redu[NW] = sab;
+        }
+        sab += hb[b];
       }
-      sab += hb;
     }
     __syncthreads();
-    const int dstar = s_star;
+    const int dstar = sh.star;
     if (dstar < 0) { found_all = false; break; }
-    prefix |= (uint32_t)dstar << sh;
-    A = redu[NW];
+    prefix |= (uint32_t)dstar << sft;
+    A = sh.redu[NW];
   }
   __syncthreads();
   if (!found_all) {
@@ -144,21 +162,33 @@ __global__ void __launch_bounds__(NT) lrfu_kernel(const DecodeParams p) {
   // ---- entries whose pbar equals the threshold key share one mass; the earliest positions win
   const uint32_t theta = prefix;
   int eq = 0;
-  for (int i = tid; i < n; i += NT) eq += (__float_as_uint(pbar[i]) == theta);
+  if (EPT > 0) {
+#pragma unroll
+    for (int k = 0; k < R; ++k)
+      if (k < kmax && tid + k * NT < n) eq += (__float_as_uint(pmr[k]) == theta);
+  } else {
+    for (int i = tid; i < n; i += NT) eq += (__float_as_uint(pbar[i]) == theta);
+  }
   eq = warp_sum_i(eq);
-  if (lane == 0) s_eq[w] = eq;
+  if (lane == 0) sh.eq[w] = eq;
   __syncthreads();
   int cnt_eq = 0;
-  for (int x = 0; x < NW; ++x) cnt_eq += s_eq[x];
-  const unsigned long long w_theta = (unsigned long long)(__uint_as_float(theta) * 1099511627776.0f);
+  for (int x = 0; x < NW; ++x) cnt_eq += sh.eq[x];
+  if (EPT > 0 && cnt_eq > 1) {   // the rank among equal keys needs every entry's key: spill them
+#pragma unroll
+    for (int k = 0; k < R; ++k)
+      if (k < kmax && tid + k * NT < n) pbar[tid + k * NT] = pmr[k];
+    __syncthreads();
+  }
+  const unsigned long long w_theta = mass_of(__uint_as_float(theta));
+
   // ---- steps 2-3: CRF/tau update; step 4 candidates
   const int k_evict = n - st.budget[uid];
   uint32_t bk0 = 0xffffffffu, bk1 = 0xffffffffu, bk2 = 0xffffffffu;
   int bidx = -1, nhit = 0;
-  for (int i = tid; i < n; i += NT) {
-    const uint32_t key = __float_as_uint(pbar[i]);
+  auto update = [&](int i, float pm, int pos_i, int tau, float crf, float dec) {
+    const uint32_t key = __float_as_uint(pm);
     bool hit = key > theta && found_all;
-    const int pos_i = st.meta_pos[mb + i];
     if (key == theta && found_all) {
       unsigned long long rank = 0;
       if (cnt_eq > 1)
@@ -166,8 +196,7 @@ __global__ void __launch_bounds__(NT) lrfu_kernel(const DecodeParams p) {
           rank += (__float_as_uint(pbar[x]) == theta) && (st.meta_pos[mb + x] < pos_i);
       hit = (A + rank * w_theta) < Pthr;
     }
-    int tau = st.meta_tau[mb + i];
-    float ct = __fmul_rn(st.tab[p.t - tau], st.meta_crf[mb + i]);
+    float ct = __fmul_rn(dec, crf);
     if (hit) {
       ct = __fadd_rn(ct, 1.0f);
       tau = p.t;
@@ -179,6 +208,30 @@ __global__ void __launch_bounds__(NT) lrfu_kernel(const DecodeParams p) {
       const uint32_t c0 = __float_as_uint(ct), c1 = (uint32_t)tau, c2 = (uint32_t)pos_i;
       const bool less = (c0 != bk0) ? (c0 < bk0) : ((c1 != bk1) ? (c1 < bk1) : (c2 < bk2));
       if (less) { bk0 = c0; bk1 = c1; bk2 = c2; bidx = i; }
+    }
+  };
+  if (EPT > 0) {
+    int pos_r[R], tau_r[R];
+    float crf_r[R], dec_r[R];
+#pragma unroll
+    for (int k = 0; k < R; ++k) {   // all loads first: they overlap
+      const int i = tid + k * NT;
+      const bool ok = k < kmax && i < n;
+      pos_r[k] = ok ? st.meta_pos[mb + i] : 0;
+      tau_r[k] = ok ? st.meta_tau[mb + i] : p.t;
+      crf_r[k] = ok ? st.meta_crf[mb + i] : 0.f;
+    }
+#pragma unroll
+    for (int k = 0; k < R; ++k) dec_r[k] = st.tab[p.t - tau_r[k]];
+#pragma unroll
+    for (int k = 0; k < R; ++k) {
+      const int i = tid + k * NT;
+      if (k < kmax && i < n) update(i, pmr[k], pos_r[k], tau_r[k], crf_r[k], dec_r[k]);
+    }
+  } else {
+    for (int i = tid; i < n; i += NT) {
+      const int tau = st.meta_tau[mb + i];
+      update(i, pbar[i], st.meta_pos[mb + i], tau, st.meta_crf[mb + i], st.tab[p.t - tau]);
     }
   }
   nhit = warp_sum_i(nhit);
@@ -194,15 +247,15 @@ __global__ void __launch_bounds__(NT) lrfu_kernel(const DecodeParams p) {
       const bool less = (o0 != bk0) ? (o0 < bk0) : ((o1 != bk1) ? (o1 < bk1) : (o2 < bk2));
       if (less) { bk0 = o0; bk1 = o1; bk2 = o2; bidx = oi; }
     }
-    if (lane == 0) { s_min[w * 4] = (int)bk0; s_min[w * 4 + 1] = (int)bk1; s_min[w * 4 + 2] = (int)bk2; s_min[w * 4 + 3] = bidx; }
+    if (lane == 0) { sh.amin[w * 4] = (int)bk0; sh.amin[w * 4 + 1] = (int)bk1; sh.amin[w * 4 + 2] = (int)bk2; sh.amin[w * 4 + 3] = bidx; }
     __syncthreads();   // also orders every CRF/tau store above before the swap below
     if (tid == 0) {
-      uint32_t a0 = (uint32_t)s_min[0], a1 = (uint32_t)s_min[1], a2 = (uint32_t)s_min[2];
-      int ai = s_min[3];
+      uint32_t a0 = (uint32_t)sh.amin[0], a1 = (uint32_t)sh.amin[1], a2 = (uint32_t)sh.amin[2];
+      int ai = sh.amin[3];
       for (int x = 1; x < NW; ++x) {
-        const uint32_t o0 = (uint32_t)s_min[x * 4], o1 = (uint32_t)s_min[x * 4 + 1], o2 = (uint32_t)s_min[x * 4 + 2];
+        const uint32_t o0 = (uint32_t)sh.amin[x * 4], o1 = (uint32_t)sh.amin[x * 4 + 1], o2 = (uint32_t)sh.amin[x * 4 + 2];
         const bool less = (o0 != a0) ? (o0 < a0) : ((o1 != a1) ? (o1 < a1) : (o2 < a2));
-        if (less) { a0 = o0; a1 = o1; a2 = o2; ai = s_min[x * 4 + 3]; }
+        if (less) { a0 = o0; a1 = o1; a2 = o2; ai = sh.amin[x * 4 + 3]; }
       }
       // the leaving entry's slot becomes the head's spare at position n-1
       if (ai != n - 1) swap_into(st, mb, ai, n - 1);
@@ -213,11 +266,27 @@ __global__ void __launch_bounds__(NT) lrfu_kernel(const DecodeParams p) {
   } else if (k_evict > 1) {
     __syncthreads();
     if (p.append && tid == 0) atomicOr(st.errword, ERR_OVER_EVICT);
-    evict_many(st, p.n_out, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh_ev,
+    evict_many(st, p.n_out, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh.ev,
                reinterpret_cast<int*>(pbar));
     n_after = n - min(k_evict, n - 1);
   }
   if (n_after == n && tid == 0) keep_and_refill(st, p.n_out, uid, seq, n, p.append != 0);
+}
+
+template <int G>
+__global__ void __launch_bounds__(NT, 4) lrfu_kernel(const DecodeParams p) {
+  __shared__ LrfuSmem sh;
+  const State& st = p.st;
+  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
+  const int uid = (seq * st.L + p.layer) * st.H + head;
+  const int n = p.n_in[uid] + p.append;
+  if (n <= 0) {
+    if (threadIdx.x == 0) p.n_out[uid] = 0;
+    return;
+  }
+  if (n <= 5 * NT) lrfu_unit<G, 5>(p, u, uid, seq, n, sh);
+  else if (n <= 17 * NT) lrfu_unit<G, 17>(p, u, uid, seq, n, sh);
+  else lrfu_unit<G, 0>(p, u, uid, seq, n, sh);
 }
 
 }  // namespace ckv
