@@ -183,6 +183,37 @@ int crystalkv_check(crystalkv_t* h, void* stream);
  */
 int crystalkv_validate(crystalkv_t* h, void* stream);
 
+/*
+ * crystalkv_validate for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a service of the library, like crystalkv_validate itself.)
+ *
+ * crystalkv_validate takes a temporary from cudaMalloc on every call.  That is not possible
+ * where a framework has already claimed all device memory for its own pool (cudaMalloc then
+ * fails although the framework has room), inside code that is being captured into a CUDA
+ * graph in a mode that forbids allocation calls, or in a serving loop that may not take the
+ * device-wide synchronisation a cudaMalloc / cudaFree pair implies.  This entry point does the
+ * same check with its per-slot counters in an array that is built into the library: it calls
+ * no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   counts_out_host  host int32[2] or NULL: [0] slot ids out of range, [1] slots not owned
+ *                    exactly once (both 0 on a sound handle)
+ *
+ * Limits and rules
+ *   - The array covers handles of at most 2^21 = 2 097 152 pool slots in total
+ *     (batch * L * H * (budget_per_head + 1 + max_answer_tokens); 1 GiB of K/V rows).  A larger
+ *     handle is refused with EINVAL and a message that says so; use crystalkv_validate there.
+ *   - Every GPU on which the library is loaded holds the array (8 MiB) until the process ends.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress,
+ *     with that device made current).  Make that first call before any stream capture begins.
+ *   - All calls on one GPU, from any handle, share the array, and it keeps the previous
+ *     call's contents; each call clears the part it uses on `stream` first.  Two calls whose
+ *     work overlaps on the GPU (different streams, no ordering between them) race: order them.
+ *   - Like crystalkv_validate it synchronises `stream` and is not for the hot path.
+ * Errors: EINVAL (NULL handle, too many slots, device ordinal above 63), ESTATE before every
+ * layer is prefilled, ECUDA, ECHECK when ownership is broken.
+ */
+int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* stream);
+
 const char* crystalkv_strerror(int code);
 const char* crystalkv_last_error(crystalkv_t* h);
 

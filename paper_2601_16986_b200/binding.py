@@ -92,6 +92,7 @@ def load_library():
     lib.crystalkv_get_counters.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
     lib.crystalkv_check.argtypes = [vp, vp]
     lib.crystalkv_validate.argtypes = [vp, vp]
+    lib.crystalkv_validate_static.argtypes = [vp, vp, vp]
     lib.crystalkv_strerror.argtypes = [i32]
     lib.crystalkv_strerror.restype = C.c_char_p
     lib.crystalkv_last_error.argtypes = [vp]
@@ -224,3 +225,10 @@ class CrystalKV:
 
     def validate(self):
         self._ck(self.lib.crystalkv_validate(self._h, _stream()))
+
+    def validate_static(self) -> np.ndarray:
+        """The same check without any device allocation (scratch built into the library; at
+        most 2**21 pool slots).  Returns int32[2]: ids out of range, slots not owned once."""
+        counts = np.full(2, -1, dtype=np.int32)
+        self._ck(self.lib.crystalkv_validate_static(self._h, counts.ctypes.data_as(C.c_void_p), _stream()))
+        return counts

@@ -668,6 +668,54 @@ int crystalkv_validate(crystalkv_t* h, void* stream) {
   return CRYSTALKV_OK;
 }
 
+// ---- the slot-ownership check for callers that cannot allocate device memory
+// The per-slot counters live in this file-scope device array instead of a temporary from
+// cudaMalloc.  Every GPU that loads the library holds the array (8 MB) until the process exits.
+constexpr long long STATIC_SEEN_SLOTS = 1ll << 21;
+static __device__ __align__(256) int g_seen_static[STATIC_SEEN_SLOTS + 2];
+constexpr int STATIC_MAX_DEVICES = 64;
+static int* g_seen_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device ordinal
+
+int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  const crystalkv_config_t& c = h->cfg;
+  for (int l = 0; l < c.n_layers; ++l)
+    if (h->t_layer[l] < 0) return fail(h, CRYSTALKV_ESTATE, "validate before every layer is prefilled");
+  const long long total = (long long)c.batch * h->slots_per_seq;
+  if (total > STATIC_SEEN_SLOTS)
+    return fail(h, CRYSTALKV_EINVAL,
+                "crystalkv_validate_static: the handle has " + std::to_string(total) + " pool slots, the built-in "
+                "scratch covers " + std::to_string(STATIC_SEEN_SLOTS) + "; use crystalkv_validate");
+  if (c.device >= STATIC_MAX_DEVICES) return fail(h, CRYSTALKV_EINVAL, "crystalkv_validate_static: device ordinal above 63");
+  CK(h, cudaSetDevice(c.device));
+  if (!g_seen_addr[c.device]) {
+    // In host code the array's name is only a handle for the runtime; its device address has
+    // to be asked for, once per device and with that device current.
+    int* addr = nullptr;
+    CK(h, cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_seen_static));
+    g_seen_addr[c.device] = addr;
+  }
+  int* seen = g_seen_addr[c.device];
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
+  // the array keeps what the last call left: everything this call reads starts from zero
+  CK(h, cudaMemsetAsync(seen, 0, (size_t)(total + 2) * sizeof(int), s));
+  mark_free_kernel<<<dim3(256, c.batch), 256, 0, s>>>(h->st, seen);
+  for (int l = 0; l < c.n_layers; ++l)
+    mark_owned_kernel<<<h->U, 128, 0, s>>>(h->st, h->st.nbuf[h->par[l]], l, seen);
+  count_bad_kernel<<<1024, 256, 0, s>>>(seen, total, seen + total + 1);
+  CK(h, cudaGetLastError());
+  int res[2] = {0, 0};
+  CK(h, cudaMemcpyAsync(res, seen + total, 2 * sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  if (counts_out_host) { counts_out_host[0] = res[0]; counts_out_host[1] = res[1]; }
+  if (res[0] || res[1])
+    return fail(h, CRYSTALKV_ECHECK, "slot ownership broken: " + std::to_string(res[0]) + " ids out of range, " +
+                                         std::to_string(res[1]) + " slots not owned exactly once");
+  return CRYSTALKV_OK;
+}
+
 int crystalkv_join(crystalkv_t* h, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
   if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
