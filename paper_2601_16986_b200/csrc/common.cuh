@@ -13,11 +13,11 @@ constexpr int GRP = 16;             // keys per streamed group (one MMA tile of 
 constexpr int NW = 8;               // warps per CTA
 constexpr int NT = NW * 32;
 constexpr int STAGES = 3;           // ring depth per warp, in groups
-constexpr int STAGE_BYTES = GRP * SLOT_BYTES;          // K tile (4 KB) then V tile (4 KB), 16-byte chunks swizzled
-constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;  // 192 KB
+constexpr int STAGE_BYTES = GRP * (SLOT_BYTES + 16);   // 16 entries, each K row + V row + 16 B of padding
+constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;  // 198 KB
 constexpr int GMIN = 4;             // fewest groups a working warp takes
 constexpr int QH = 8;               // query heads of a group as padded for the MMA N dimension
-constexpr int MAX_UNITS_PER_CALL = 4096;
+constexpr int MAX_UNITS_PER_CALL = 2048;   // bounded by the split tables in shared memory
 constexpr int NSETS = 3;            // scratch sets cycled by consecutive launches
 
 // error word bits raised by device-side consistency checks (never a trap)
@@ -25,6 +25,7 @@ constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence
 constexpr int ERR_OVER_EVICT = 2;       // a decode step found a head more than one entry over budget
 constexpr int ERR_CAPACITY = 4;         // a head's list would outgrow its capacity
 constexpr int ERR_NUCLEUS = 8;          // the top-p threshold search did not find its boundary
+constexpr int ERR_COPY_TIMEOUT = 16;    // a bulk copy into shared memory did not complete within a second
 
 struct State {
   // K/V pool: [batch][slots_per_seq][512 B]

@@ -135,7 +135,7 @@ int validate(const crystalkv_config_t* c, std::string& why) {
   if (c->n_layers < 1 || c->n_kv_heads < 1 || c->batch < 1) { why = "n_layers, n_kv_heads, batch must be >= 1"; return CRYSTALKV_EINVAL; }
   if (c->n_q_heads < c->n_kv_heads || c->n_q_heads % c->n_kv_heads) { why = "n_q_heads must be a multiple of n_kv_heads"; return CRYSTALKV_EINVAL; }
   if (c->n_q_heads / c->n_kv_heads > 8) { why = "group size above 8"; return CRYSTALKV_EINVAL; }
-  if ((long long)c->batch * c->n_kv_heads > MAX_UNITS_PER_CALL) { why = "batch * n_kv_heads above 4096"; return CRYSTALKV_EINVAL; }
+  if ((long long)c->batch * c->n_kv_heads > MAX_UNITS_PER_CALL) { why = "batch * n_kv_heads above 2048"; return CRYSTALKV_EINVAL; }
   if (c->mode != CRYSTALKV_MODE_EVICT && c->mode != CRYSTALKV_MODE_FULLKV) { why = "bad mode"; return CRYSTALKV_EINVAL; }
   if (c->max_context < 2) { why = "max_context must be >= 2"; return CRYSTALKV_EINVAL; }
   if (c->mode == CRYSTALKV_MODE_EVICT && c->budget_per_head < 1) { why = "budget_per_head must be >= 1"; return CRYSTALKV_EINVAL; }
@@ -311,7 +311,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   cudaDeviceProp prop;
   CKC(cudaGetDeviceProperties(&prop, c.device));
   h->num_sms = prop.multiProcessorCount;
-  h->smem = RING_BYTES + (size_t)(2 * h->U + 1) * sizeof(int);
+  h->smem = RING_BYTES + NW * STAGES * 8 + (size_t)(2 * h->U + 1) * sizeof(int);
   int bps = 0;
   CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem));
   CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
@@ -736,6 +736,7 @@ int crystalkv_check(crystalkv_t* h, void* stream) {
   if (w & ERR_OVER_EVICT) msg += " head more than one entry over budget in a decode step;";
   if (w & ERR_CAPACITY) msg += " head list capacity exceeded;";
   if (w & ERR_NUCLEUS) msg += " top-p boundary not found;";
+  if (w & ERR_COPY_TIMEOUT) msg += " a bulk copy into shared memory timed out;";
   return fail(h, CRYSTALKV_ECHECK, msg);
 }
 
