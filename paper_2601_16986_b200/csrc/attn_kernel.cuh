@@ -119,6 +119,46 @@ __device__ __forceinline__ void merge_rows(const float* pbase, int PS, int npiec
     }
 }
 
+// The whole merge of HB heads over at most PB pieces in one round of loads: every lane loads
+// the pieces' (m, l) itself (broadcast loads) next to its 4 channels of every O row, so nothing
+// waits for a header round.  mm, L: merged reference point and normaliser per head.
+template <int HB, int PB>
+__device__ __forceinline__ void merge_small(const float* pbase, int PS, int npieces, int g0, int G, int lane,
+                                            float (&mm)[HB], float (&L)[HB], float4 (&acc)[HB]) {
+  float4 v[HB][PB];
+  float pm[HB][PB], pl[HB][PB];
+#pragma unroll
+  for (int j = 0; j < PB; ++j) {
+    const bool okp = j < npieces;
+    const float* pp = pbase + (size_t)j * PS;
+#pragma unroll
+    for (int h = 0; h < HB; ++h) {
+      const bool ok = okp && g0 + h < G;
+      pm[h][j] = ok ? __ldcg(pp + g0 + h) : -INFINITY;
+      pl[h][j] = ok ? __ldcg(pp + 8 + g0 + h) : 0.f;
+      v[h][j] = ok ? __ldcg(reinterpret_cast<const float4*>(pp + 16 + (g0 + h) * HD) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < HB; ++h) {
+    float m = pm[h][0];
+#pragma unroll
+    for (int j = 1; j < PB; ++j) m = fmaxf(m, pm[h][j]);
+    mm[h] = m;
+    float l = 0.f;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < PB; ++j) {
+      const float c = (pm[h][j] > -INFINITY) ? ex2(pm[h][j] - m) : 0.f;
+      l = fmaf(pl[h][j], c, l);
+      a.x = fmaf(v[h][j].x, c, a.x); a.y = fmaf(v[h][j].y, c, a.y);
+      a.z = fmaf(v[h][j].z, c, a.z); a.w = fmaf(v[h][j].w, c, a.w);
+    }
+    L[h] = l;
+    acc[h] = a;
+  }
+}
+
 __global__ void __maxnreg__(192) attn_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const State& st = p.st;
@@ -400,58 +440,68 @@ __global__ void __maxnreg__(192) attn_kernel(const DecodeParams p) {
     // so its time is the number of dependent load rounds: loads go out in batches before anything
     // consumes them.
     const float* pbase = p.sc.partials + (size_t)u * p.sc.pmax * PS;
-    const int hh = lane & 7, pl = lane >> 3;   // header phase: lane = (piece mod 4, head)
-    float mm = -INFINITY, Ls = 0.f;
-    for (int pc0 = 0; pc0 < npieces; pc0 += 8) {
-      const int pa = pc0 + pl, pb = pc0 + pl + 4;
-      const bool oa = pa < npieces, ob = pb < npieces;
-      const float ma = oa ? __ldcg(pbase + (size_t)pa * PS + hh) : -INFINITY;
-      const float mb_ = ob ? __ldcg(pbase + (size_t)pb * PS + hh) : -INFINITY;
-      const float la = oa ? __ldcg(pbase + (size_t)pa * PS + 8 + hh) : 0.f;
-      const float lb = ob ? __ldcg(pbase + (size_t)pb * PS + 8 + hh) : 0.f;
-      const float mn = fmaxf(mm, fmaxf(ma, mb_));
-      if (mn > -INFINITY) Ls = Ls * ex2(mm - mn) + la * ex2(ma - mn) + lb * ex2(mb_ - mn);   // ex2(-inf) = 0 covers the gaps
-      mm = mn;
-    }
-#pragma unroll
-    for (int x = 8; x < 32; x <<= 1) {   // combine the four piece classes
-      const float mo = __shfl_xor_sync(0xffffffffu, mm, x), lo_ = __shfl_xor_sync(0xffffffffu, Ls, x);
-      const float mn = fmaxf(mm, mo);
-      if (mn > -INFINITY) Ls = Ls * ex2(mm - mn) + lo_ * ex2(mo - mn);
-      mm = mn;
-    }
-    if (lane < G && p.track) {   // reference point and normaliser of the step's softmax, for the LRFU kernel
-      p.sc.mfin[u * (2 * QH) + lane] = mm;
-      p.sc.mfin[u * (2 * QH) + QH + lane] = Ls;
-    }
-    auto store_out = [&](int g, const float4& a) {
-      const float iv = 1.0f / __shfl_sync(0xffffffffu, Ls, g);
+    auto put = [&](int g, float m, float L, const float4& a) {   // one head's result
       if (g < G) {
+        const float iv = 1.0f / L;
         uint2 pk;
         pk.x = pack_bf16(a.x * iv, a.y * iv);
         pk.y = pack_bf16(a.z * iv, a.w * iv);
         *reinterpret_cast<uint2*>(p.out + ((size_t)(u * G + g)) * HD + lane * 4) = pk;
+        if (lane == 0 && p.track) {   // reference point and normaliser of the step's softmax, for the LRFU kernel
+          p.sc.mfin[u * (2 * QH) + g] = m;
+          p.sc.mfin[u * (2 * QH) + QH + g] = L;
+        }
       }
     };
-    if (npieces <= 4) {   // the usual case: four heads x four pieces per round
-      for (int g0 = 0; g0 < G; g0 += 4) {
-        float mg[4];
-        float4 acc[4];
+    if (npieces <= 4) {   // the usual case: one round of loads for up to five heads
+      if (G <= 5) {
+        float mm[5], L[5];
+        float4 acc[5];
+        merge_small<5, 4>(pbase, PS, npieces, 0, G, lane, mm, L, acc);
 #pragma unroll
-        for (int h = 0; h < 4; ++h) { mg[h] = __shfl_sync(0xffffffffu, mm, (g0 + h) & 7); acc[h] = make_float4(0.f, 0.f, 0.f, 0.f); }
-        merge_rows<4, 4>(pbase, PS, npieces, 0, g0, G, lane, mg, acc);
+        for (int h = 0; h < 5; ++h) put(h, mm[h], L[h], acc[h]);
+      } else {
+        for (int g0 = 0; g0 < G; g0 += 4) {
+          float mm[4], L[4];
+          float4 acc[4];
+          merge_small<4, 4>(pbase, PS, npieces, g0, G, lane, mm, L, acc);
 #pragma unroll
-        for (int h = 0; h < 4; ++h) store_out(g0 + h, acc[h]);
+          for (int h = 0; h < 4; ++h) put(g0 + h, mm[h], L[h], acc[h]);
+        }
       }
     } else {
+      const int hh = lane & 7, pl = lane >> 3;   // header phase: lane = (piece mod 4, head)
+      float mm = -INFINITY, Ls = 0.f;
+      for (int pc0 = 0; pc0 < npieces; pc0 += 8) {
+        const int pa = pc0 + pl, pb = pc0 + pl + 4;
+        const bool oa = pa < npieces, ob = pb < npieces;
+        const float ma = oa ? __ldcg(pbase + (size_t)pa * PS + hh) : -INFINITY;
+        const float mb_ = ob ? __ldcg(pbase + (size_t)pb * PS + hh) : -INFINITY;
+        const float la = oa ? __ldcg(pbase + (size_t)pa * PS + 8 + hh) : 0.f;
+        const float lb = ob ? __ldcg(pbase + (size_t)pb * PS + 8 + hh) : 0.f;
+        const float mn = fmaxf(mm, fmaxf(ma, mb_));
+        if (mn > -INFINITY) Ls = Ls * ex2(mm - mn) + la * ex2(ma - mn) + lb * ex2(mb_ - mn);   // ex2(-inf) = 0 covers the gaps
+        mm = mn;
+      }
+#pragma unroll
+      for (int x = 8; x < 32; x <<= 1) {   // combine the four piece classes
+        const float mo = __shfl_xor_sync(0xffffffffu, mm, x), lo_ = __shfl_xor_sync(0xffffffffu, Ls, x);
+        const float mn = fmaxf(mm, mo);
+        if (mn > -INFINITY) Ls = Ls * ex2(mm - mn) + lo_ * ex2(mo - mn);
+        mm = mn;
+      }
       for (int g0 = 0; g0 < G; g0 += 2) {
-        float mg[2];
+        float mg[2], Lg[2];
         float4 acc[2];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) { mg[h] = __shfl_sync(0xffffffffu, mm, (g0 + h) & 7); acc[h] = make_float4(0.f, 0.f, 0.f, 0.f); }
+        for (int h = 0; h < 2; ++h) {
+          mg[h] = __shfl_sync(0xffffffffu, mm, (g0 + h) & 7);
+          Lg[h] = __shfl_sync(0xffffffffu, Ls, (g0 + h) & 7);
+          acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         for (int pc0 = 0; pc0 < npieces; pc0 += 8) merge_rows<2, 8>(pbase, PS, npieces, pc0, g0, G, lane, mg, acc);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) store_out(g0 + h, acc[h]);
+        for (int h = 0; h < 2; ++h) put(g0 + h, mg[h], Lg[h], acc[h]);
       }
     }
     if (lane == 0) {

@@ -3,7 +3,10 @@
 //   step 1   softmax weights per query head from the logits, the attention kernel's merged
 //            reference point and normaliser (accurate expf), group-mean probability pbar,
 //            hit mask = smallest descending-pbar prefix whose exclusive mass is below p
-//            (equal pbar: ascending position);
+//            (equal pbar: ascending position).  The threshold value is found exactly: one
+//            histogram of 1024 bins of 1/64 octave around 1/n locates its bin, the few
+//            entries of that bin are ranked against one another; a bin outside the window
+//            or with more than 64 entries falls back to three radix passes over all bits;
 //   step 2-3 hits: CRF <- lambda^(t - tau) CRF + 1, tau <- t; misses only get the decayed
 //            CRF_temp, which is not stored;
 //   step 4   the entries lowest under (CRF_temp, tau, position) leave until the head is
@@ -19,10 +22,19 @@ namespace ckv {
 constexpr int HIST_BINS = 2048;
 constexpr float MASS_ONE = 1099511627776.0f;   // 2^40
 
+constexpr int FINE_BINS = 1024;   // fast path: bins of 2^17 key steps = 1/64 octave, 16 octaves wide
+constexpr int FINE_SHIFT = 17;
+constexpr int MAX_CAND = 64;
+
 struct LrfuSmem {
   unsigned hist_lo[HIST_BINS];   // per-bin mass, low 16 bits of every term
   unsigned hist_hi[HIST_BINS];   // per-bin mass, the bits above
   unsigned long long redu[NW + 4];
+  unsigned cand[MAX_CAND];       // keys of the entries in the threshold's bin
+  unsigned long long A_theta;    // fast path result: mass strictly above the threshold key
+  unsigned theta;                //                   the threshold key
+  int cnt_theta;                 //                   entries that carry it
+  int ncand;
   int star;
   int eq[NW];
   int amin[NW * 4];
@@ -61,7 +73,6 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     return pm;
   };
   float pmr[R];
-  unsigned long long wsum = 0;
   if (EPT > 0) {
 #pragma unroll
     for (int k = 0; k < R; ++k) {
@@ -69,45 +80,26 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       pmr[k] = 0.f;
       if (k < kmax && i < n) {
         pmr[k] = pbar_of(i);
-        wsum += mass_of(pmr[k]);
       }
     }
   } else {
     for (int i = tid; i < n; i += NT) {
-      const float pm = pbar_of(i);
-      pbar[i] = pm;
-      wsum += mass_of(pm);
+      pbar[i] = pbar_of(i);
     }
   }
-  wsum = warp_sum_u64(wsum);
-  if (lane == 0) sh.redu[w] = wsum;
+  // ---- fast path, pass over all entries: histogram of mass in fine bins around 1/n
+  //      bin(key) = clamp((key >> 17) - base, 0, 1023), monotone in key
+  const int fbase = (int)(__float_as_uint(1.0f / (256.0f * (float)n)) >> FINE_SHIFT);
+  auto fbin = [&](uint32_t key) { return min(FINE_BINS - 1, max(0, (int)(key >> FINE_SHIFT) - fbase)); };
+  for (int b = tid; b < FINE_BINS; b += NT) { sh.hist_lo[b] = 0u; sh.hist_hi[b] = 0u; }
+  if (tid == 0) { sh.star = -1; sh.ncand = 0; sh.theta = 0xffffffffu; sh.cnt_theta = 0; }
   __syncthreads();
-  unsigned long long W = 0;
-  for (int x = 0; x < NW; ++x) W += sh.redu[x];
-  // hit  <=>  mass strictly before the entry  <  p * W
-  const unsigned long long Pthr = (unsigned long long)ceil((double)p.top_p * (double)W);
-
-  // ---- threshold key by MSB-first radix passes over the fp32 bits of pbar (11, 11, 10 bits)
-  unsigned long long A = 0;   // mass of keys strictly above the current prefix range
-  uint32_t prefix = 0;
-  bool found_all = true;
-  for (int pass = 0; pass < 3; ++pass) {
-    const int sft = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-    const int wid = pass == 2 ? 10 : 11;
-    const int nb = 1 << wid;
-    __syncthreads();
-    for (int b = tid; b < nb; b += NT) { sh.hist_lo[b] = 0u; sh.hist_hi[b] = 0u; }
-    if (tid == 0) sh.star = -1;
-    __syncthreads();
+  {
     auto add = [&](float pm) {
-      const uint32_t key = __float_as_uint(pm);
-      const bool match = (pass == 0) || ((key >> (sft + wid)) == (prefix >> (sft + wid)));
-      if (match) {
-        const unsigned long long m = mass_of(pm);
-        const int b = (key >> sft) & (nb - 1);
-        atomicAdd(&sh.hist_lo[b], (unsigned)(m & 0xffffu));
-        atomicAdd(&sh.hist_hi[b], (unsigned)(m >> 16));
-      }
+      const unsigned long long m = mass_of(pm);
+      const int b = fbin(__float_as_uint(pm));
+      atomicAdd(&sh.hist_lo[b], (unsigned)(m & 0xffffu));
+      atomicAdd(&sh.hist_hi[b], (unsigned)(m >> 16));
     };
     if (EPT > 0) {
 #pragma unroll
@@ -116,15 +108,17 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     } else {
       for (int i = tid; i < n; i += NT) add(pbar[i]);
     }
-    __syncthreads();
-    // suffix sums from the top bin: thread k owns bins [k*per, (k+1)*per)
-    const int per = nb / NT;
-    unsigned long long hb[HIST_BINS / NT];
-    unsigned long long loc = 0;
+  }
+  __syncthreads();
+  unsigned long long W, Pthr;
+  unsigned long long A = 0;   // mass of keys strictly above the threshold's bin / prefix range
+  {
+    // suffix sums from the top bin: thread k owns bins [4k, 4k + 4)
+    constexpr int PER = FINE_BINS / NT;
+    unsigned long long hb[PER], loc = 0;
 #pragma unroll
-    for (int b = 0; b < HIST_BINS / NT; ++b) {
-      hb[b] = 0;
-      if (b < per) hb[b] = ((unsigned long long)sh.hist_hi[tid * per + b] << 16) + sh.hist_lo[tid * per + b];
+    for (int b = 0; b < PER; ++b) {
+      hb[b] = ((unsigned long long)sh.hist_hi[tid * PER + b] << 16) + sh.hist_lo[tid * PER + b];
       loc += hb[b];
     }
     unsigned long long suf = loc;   // inclusive suffix scan across the warp (higher lane = higher bins)
@@ -136,44 +130,162 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     if (lane == 0) sh.redu[w] = suf;
     __syncthreads();
     unsigned long long above = 0;
-    for (int x = w + 1; x < NW; ++x) above += sh.redu[x];
-    unsigned long long sab = A + above + (suf - loc);   // mass above this thread's top bin
+    W = 0;
+    for (int x = 0; x < NW; ++x) {
+      const unsigned long long r = sh.redu[x];
+      W += r;
+      if (x > w) above += r;
+    }
+    // hit  <=>  mass strictly before the entry  <  p * W
+    Pthr = (unsigned long long)ceil((double)p.top_p * (double)W);
+    unsigned long long sab = above + (suf - loc);   // mass above this thread's top bin
 #pragma unroll
-    for (int b = HIST_BINS / NT - 1; b >= 0; --b) {
-      if (b < per) {
-        if (sab < Pthr && Pthr <= sab + hb[b]) {
-          sh.star = tid * per + b;
-          sh.redu[NW] = sab;
-        }
-        sab += hb[b];
+    for (int b = PER - 1; b >= 0; --b) {
+      if (sab < Pthr && Pthr <= sab + hb[b]) {
+        sh.star = tid * PER + b;
+        sh.redu[NW] = sab;
       }
+      sab += hb[b];
     }
     __syncthreads();
-    const int dstar = sh.star;
-    if (dstar < 0) { found_all = false; break; }
-    prefix |= (uint32_t)dstar << sft;
-    A = sh.redu[NW];
   }
-  __syncthreads();
-  if (!found_all) {
-    if (tid == 0) atomicOr(st.errword, ERR_NUCLEUS);
-    prefix = 0xffffffffu;  // nothing is a hit
-  }
-  // ---- entries whose pbar equals the threshold key share one mass; the earliest positions win
-  const uint32_t theta = prefix;
-  int eq = 0;
-  if (EPT > 0) {
-#pragma unroll
-    for (int k = 0; k < R; ++k)
-      if (k < kmax && tid + k * NT < n) eq += (__float_as_uint(pmr[k]) == theta);
-  } else {
-    for (int i = tid; i < n; i += NT) eq += (__float_as_uint(pbar[i]) == theta);
-  }
-  eq = warp_sum_i(eq);
-  if (lane == 0) sh.eq[w] = eq;
-  __syncthreads();
+  uint32_t theta = 0xffffffffu;
   int cnt_eq = 0;
-  for (int x = 0; x < NW; ++x) cnt_eq += sh.eq[x];
+  bool found_all = false;
+  const int bstar = sh.star;
+  if (bstar > 0 && bstar < FINE_BINS - 1) {   // inside the window: rank the bin's entries exactly
+    A = sh.redu[NW];
+    auto offer = [&](float pm) {
+      const uint32_t key = __float_as_uint(pm);
+      if (fbin(key) == bstar) {
+        const int x = atomicAdd(&sh.ncand, 1);
+        if (x < MAX_CAND) sh.cand[x] = key;
+      }
+    };
+    if (EPT > 0) {
+#pragma unroll
+      for (int k = 0; k < R; ++k)
+        if (k < kmax && tid + k * NT < n) offer(pmr[k]);
+    } else {
+      for (int i = tid; i < n; i += NT) offer(pbar[i]);
+    }
+    __syncthreads();
+    const int c = sh.ncand;
+    if (c <= MAX_CAND) {
+      // candidate x carries the threshold iff  A + mass(keys above it) < Pthr <= that + mass(keys equal)
+      if (tid < c) {
+        const uint32_t mine = sh.cand[tid];
+        const unsigned long long wm = mass_of(__uint_as_float(mine));
+        unsigned long long gt = 0;
+        int eqc = 0;
+        for (int x = 0; x < c; ++x) {
+          const uint32_t kx = sh.cand[x];
+          if (kx > mine) gt += mass_of(__uint_as_float(kx));
+          eqc += (kx == mine);
+        }
+        if (A + gt < Pthr && Pthr <= A + gt + (unsigned long long)eqc * wm) {
+          sh.theta = mine;            // every carrier writes the same three values
+          sh.A_theta = A + gt;
+          sh.cnt_theta = eqc;
+        }
+      }
+      __syncthreads();
+      if (sh.cnt_theta > 0) {
+        theta = sh.theta;
+        A = sh.A_theta;
+        cnt_eq = sh.cnt_theta;
+        found_all = true;
+      }
+    }
+  }
+  if (!found_all) {
+    // ---- general path: MSB-first radix passes over the fp32 bits of pbar (11, 11, 10 bits)
+    A = 0;
+    uint32_t prefix = 0;
+    found_all = true;
+    for (int pass = 0; pass < 3; ++pass) {
+      const int sft = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+      const int wid = pass == 2 ? 10 : 11;
+      const int nb = 1 << wid;
+      __syncthreads();
+      for (int b = tid; b < nb; b += NT) { sh.hist_lo[b] = 0u; sh.hist_hi[b] = 0u; }
+      if (tid == 0) sh.star = -1;
+      __syncthreads();
+      auto add = [&](float pm) {
+        const uint32_t key = __float_as_uint(pm);
+        const bool match = (pass == 0) || ((key >> (sft + wid)) == (prefix >> (sft + wid)));
+        if (match) {
+          const unsigned long long m = mass_of(pm);
+          const int b = (key >> sft) & (nb - 1);
+          atomicAdd(&sh.hist_lo[b], (unsigned)(m & 0xffffu));
+          atomicAdd(&sh.hist_hi[b], (unsigned)(m >> 16));
+        }
+      };
+      if (EPT > 0) {
+#pragma unroll
+        for (int k = 0; k < R; ++k)
+          if (k < kmax && tid + k * NT < n) add(pmr[k]);
+      } else {
+        for (int i = tid; i < n; i += NT) add(pbar[i]);
+      }
+      __syncthreads();
+      // suffix sums from the top bin: thread k owns bins [k*per, (k+1)*per)
+      const int per = nb / NT;
+      unsigned long long hb[HIST_BINS / NT];
+      unsigned long long loc = 0;
+#pragma unroll
+      for (int b = 0; b < HIST_BINS / NT; ++b) {
+        hb[b] = 0;
+        if (b < per) hb[b] = ((unsigned long long)sh.hist_hi[tid * per + b] << 16) + sh.hist_lo[tid * per + b];
+        loc += hb[b];
+      }
+      unsigned long long suf = loc;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long x = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += x;
+      }
+      if (lane == 0) sh.redu[w] = suf;
+      __syncthreads();
+      unsigned long long above = 0;
+      for (int x = w + 1; x < NW; ++x) above += sh.redu[x];
+      unsigned long long sab = A + above + (suf - loc);   // mass above this thread's top bin
+#pragma unroll
+      for (int b = HIST_BINS / NT - 1; b >= 0; --b) {
+        if (b < per) {
+          if (sab < Pthr && Pthr <= sab + hb[b]) {
+            sh.star = tid * per + b;
+            sh.redu[NW] = sab;
+          }
+          sab += hb[b];
+        }
+      }
+      __syncthreads();
+      const int dstar = sh.star;
+      if (dstar < 0) { found_all = false; break; }
+      prefix |= (uint32_t)dstar << sft;
+      A = sh.redu[NW];
+    }
+    __syncthreads();
+    if (!found_all) {
+      if (tid == 0) atomicOr(st.errword, ERR_NUCLEUS);
+      prefix = 0xffffffffu;  // nothing is a hit
+    }
+    // entries whose pbar equals the threshold key share one mass; the earliest positions win
+    theta = prefix;
+    int eq = 0;
+    if (EPT > 0) {
+#pragma unroll
+      for (int k = 0; k < R; ++k)
+        if (k < kmax && tid + k * NT < n) eq += (__float_as_uint(pmr[k]) == theta);
+    } else {
+      for (int i = tid; i < n; i += NT) eq += (__float_as_uint(pbar[i]) == theta);
+    }
+    eq = warp_sum_i(eq);
+    if (lane == 0) sh.eq[w] = eq;
+    __syncthreads();
+    for (int x = 0; x < NW; ++x) cnt_eq += sh.eq[x];
+  }
   if (EPT > 0 && cnt_eq > 1) {   // the rank among equal keys needs every entry's key: spill them
 #pragma unroll
     for (int k = 0; k < R; ++k)
