@@ -159,7 +159,7 @@ __device__ __forceinline__ void merge_small(const float* pbase, int PS, int npie
   }
 }
 
-__global__ void __maxnreg__(192) attn_kernel(const DecodeParams p) {
+__global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const State& st = p.st;
   // Without `early` the kernel before this one may still be writing the lists this one reads.

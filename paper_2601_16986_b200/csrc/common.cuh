@@ -18,7 +18,7 @@ constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;  // 198 KB
 constexpr int GMIN = 4;             // fewest groups a working warp takes
 constexpr int QH = 8;               // query heads of a group as padded for the MMA N dimension
 constexpr int MAX_UNITS_PER_CALL = 2048;   // bounded by the split tables in shared memory
-constexpr int NSETS = 3;            // scratch sets cycled by consecutive launches
+constexpr int NSETS = 8;            // logit scratch sets cycled by consecutive tracked launches
 
 // error word bits raised by device-side consistency checks (never a trap)
 constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence's free list was empty
@@ -46,7 +46,8 @@ struct State {
   int batch, L, H, cap;
 };
 
-// scratch of one launch pair (attention kernel, then LRFU kernel); NSETS sets are cycled
+// scratch of one launch pair (attention kernel, then LRFU kernel), assembled per launch: the
+// logits and (m, l) come from one of NSETS cycled sets, the partials and tickets from one of two
 struct Scratch {
   float* logits;     // [U][cap_s][QH] scaled logits of the step, one 32-byte row per entry
   float* pbar;       // [U][cap_s] group-mean probabilities (reused as int scratch)

@@ -30,10 +30,19 @@ struct crystalkv {
   size_t smem = 0;
   long long slots_per_seq = 0;
   State st{};
-  Scratch sc[NSETS]{};
+  // scratch: logits and merged (m, l) per cycled set (the LRFU kernel reads them while later
+  // attention kernels run), partials and tickets alternate between two (attention kernels do
+  // not overlap one another's compute), pbar is only touched by kernels that run one at a time
+  float* sc_logits[NSETS] = {};
+  float* sc_mfin[NSETS] = {};
+  float* sc_partials[2] = {};
+  int* sc_ticket[2] = {};
+  float* sc_pbar = nullptr;
+  int cap_s = 0, pmax = 0;
+  long long nA = 0;                // attention launches so far
   std::vector<int> t_layer, par;   // per layer: time of the last step, current count buffer
   // LRFU launches are numbered; launch k uses scratch set k % NSETS and event k % EV_RING
-  static constexpr int EV_RING = 8;
+  static constexpr int EV_RING = 16;
   cudaStream_t side = nullptr;
   cudaEvent_t evA = nullptr, evF[EV_RING] = {};
   long long kF = 0, joined = -1;
@@ -167,7 +176,15 @@ int check_unit(crystalkv_t* h, int layer, int seq, int head) {
 DecodeParams make_params(crystalkv_t* h, int layer, int set) {
   DecodeParams p{};
   p.st = h->st;
-  p.sc = h->sc[set];
+  (void)set;
+  p.sc.cap_s = h->cap_s;
+  p.sc.pmax = h->pmax;
+  p.sc.pbar = h->sc_pbar;
+  p.sc.partials = h->sc_partials[h->nA & 1];
+  p.sc.ticket = h->sc_ticket[h->nA & 1];
+  p.sc.logits = h->sc_logits[0];
+  p.sc.mfin = h->sc_mfin[0];
+  h->nA++;
   p.layer = layer;
   p.G = h->G;
   p.n_in = h->st.nbuf[h->par[layer]];
@@ -193,12 +210,17 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
   if (track) {
     // launch k reuses the scratch of launch k - NSETS and continues the state its layer's
     // previous LRFU launch wrote; the internal stream runs in order, so one event covers both
+    // A wait on the caller's stream costs several microseconds (the attention kernel behind it
+    // no longer starts early), so one wait covers as many launches as the sets allow: it targets
+    // the newest LRFU launch that has had two attention kernels' time to finish.
     const long long need = std::max(k - NSETS, h->lastF[layer]);
     if (need >= 0 && need > h->joined) {
-      CK(h, cudaStreamWaitEvent(s, h->evF[need % crystalkv::EV_RING], 0));
-      h->joined = need;
+      const long long target = std::max(need, k - 3);
+      CK(h, cudaStreamWaitEvent(s, h->evF[target % crystalkv::EV_RING], 0));
+      h->joined = target;
     }
-    p.sc = h->sc[k % NSETS];
+    p.sc.logits = h->sc_logits[k % NSETS];
+    p.sc.mfin = h->sc_mfin[k % NSETS];
   }
   // The attention kernel may start while the kernel ahead of it still runs: it first fills its
   // pipeline from the cache and waits for that kernel before it touches the call's inputs.
@@ -340,17 +362,18 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   DA(&st.counters, 4);
   DA(&h->Asum, h->units);
   const int capgroups = (h->cap + GRP - 1) / GRP;
+  h->cap_s = evict ? h->cap : 1;
+  h->pmax = capgroups / GMIN + 2;
   for (int i = 0; i < NSETS; ++i) {
-    Scratch& sc = h->sc[i];
-    sc.cap_s = evict ? h->cap : 1;
-    sc.pmax = capgroups / GMIN + 2;
-    DA(&sc.logits, (size_t)h->U * sc.cap_s * QH);
-    DA(&sc.pbar, (size_t)h->U * sc.cap_s);
-    DA(&sc.partials, (size_t)h->U * sc.pmax * (16 + h->G * HD));
-    DA(&sc.mfin, (size_t)h->U * 2 * QH);
-    DA(&sc.ticket, h->U);
-    CKC(cudaMemset(sc.ticket, 0, (size_t)h->U * sizeof(int)));
+    DA(&h->sc_logits[i], (size_t)h->U * h->cap_s * QH);
+    DA(&h->sc_mfin[i], (size_t)h->U * 2 * QH);
   }
+  for (int i = 0; i < 2; ++i) {
+    DA(&h->sc_partials[i], (size_t)h->U * h->pmax * (16 + h->G * HD));
+    DA(&h->sc_ticket[i], h->U);
+    CKC(cudaMemset(h->sc_ticket[i], 0, (size_t)h->U * sizeof(int)));
+  }
+  DA(&h->sc_pbar, (size_t)h->U * h->cap_s);
   const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
   DA(&h->dq, qn); DA(&h->dout, qn); DA(&h->dk, kn); DA(&h->dv, kn); DA(&h->dummy_out, qn);
 
@@ -499,9 +522,8 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   const long long B_total = (long long)c.budget_per_head * N;
   alg2_kernel<<<c.batch, NT, sm, s>>>(h->Asum, h->st.budget, c.n_layers, c.n_kv_heads, B_total, c.min_budget, c.max_budget);
   CK(h, cudaGetLastError());
-  const Scratch& sc = h->sc[0];
   for (int l = 0; l < c.n_layers; ++l) {
-    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, n_cur, l, t_last, reinterpret_cast<int*>(sc.pbar), sc.cap_s);
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, n_cur, l, t_last, reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
     CK(h, cudaGetLastError());
   }
   return CRYSTALKV_OK;
@@ -519,9 +541,8 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
   CK(h, cudaMemcpyAsync(h->st.budget + uid, &budget, sizeof(int), cudaMemcpyHostToDevice, s));
   CK(h, cudaStreamSynchronize(s));
   if (h->t_layer[layer] >= 0) {
-    const Scratch& sc = h->sc[0];
     shrink_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer, h->t_layer[layer],
-                                      reinterpret_cast<int*>(sc.pbar), sc.cap_s);
+                                      reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
     CK(h, cudaGetLastError());
   }
   return CRYSTALKV_OK;

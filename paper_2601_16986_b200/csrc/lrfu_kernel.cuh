@@ -73,19 +73,32 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     return pm;
   };
   float pmr[R];
-  if (EPT > 0) {
+  if (EPT > 0 && EPT <= 8) {
+    // all logit rows first (clamped index, no branch), so that their latencies overlap
+    float4 ra[R], rb[R];
+#pragma unroll
+    for (int k = 0; k < R; ++k) {
+      const int i = min(tid + k * NT, n - 1);
+      ra[k] = *reinterpret_cast<const float4*>(S + (size_t)i * QH);
+      rb[k] = (G > 4) ? *reinterpret_cast<const float4*>(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int k = 0; k < R; ++k) {
+      const float sv[8] = {ra[k].x, ra[k].y, ra[k].z, ra[k].w, rb[k].x, rb[k].y, rb[k].z, rb[k].w};
+      float pm = 0.f;
+#pragma unroll
+      for (int g = 0; g < G; ++g) pm = fmaf(expf(sv[g] - mx[g]), invl[g], pm);
+      pmr[k] = (tid + k * NT < n) ? pm : 0.f;
+    }
+  } else if (EPT > 0) {
 #pragma unroll
     for (int k = 0; k < R; ++k) {
       const int i = tid + k * NT;
       pmr[k] = 0.f;
-      if (k < kmax && i < n) {
-        pmr[k] = pbar_of(i);
-      }
+      if (k < kmax && i < n) pmr[k] = pbar_of(i);
     }
   } else {
-    for (int i = tid; i < n; i += NT) {
-      pbar[i] = pbar_of(i);
-    }
+    for (int i = tid; i < n; i += NT) pbar[i] = pbar_of(i);
   }
   // ---- fast path, pass over all entries: histogram of mass in fine bins around 1/n
   //      bin(key) = clamp((key >> 17) - base, 0, 1023), monotone in key
@@ -322,7 +335,16 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       if (less) { bk0 = c0; bk1 = c1; bk2 = c2; bidx = i; }
     }
   };
-  if (EPT > 0) {
+  if (EPT > 8) {   // many entries per thread: one at a time keeps the registers down
+#pragma unroll
+    for (int k = 0; k < R; ++k) {
+      const int i = tid + k * NT;
+      if (k < kmax && i < n) {
+        const int tau = st.meta_tau[mb + i];
+        update(i, pmr[k], st.meta_pos[mb + i], tau, st.meta_crf[mb + i], __ldg(st.tab + (p.t - tau)));
+      }
+    }
+  } else if (EPT > 0) {
     int pos_r[R], tau_r[R];
     float crf_r[R], dec_r[R];
 #pragma unroll
@@ -334,7 +356,7 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       crf_r[k] = ok ? st.meta_crf[mb + i] : 0.f;
     }
 #pragma unroll
-    for (int k = 0; k < R; ++k) dec_r[k] = st.tab[p.t - tau_r[k]];
+    for (int k = 0; k < R; ++k) dec_r[k] = __ldg(st.tab + (p.t - tau_r[k]));
 #pragma unroll
     for (int k = 0; k < R; ++k) {
       const int i = tid + k * NT;
@@ -386,7 +408,7 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
 }
 
 template <int G>
-__global__ void __launch_bounds__(NT, 4) lrfu_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
   __shared__ LrfuSmem sh;
   const State& st = p.st;
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
