@@ -6,7 +6,7 @@
 //            (equal pbar: ascending position).  The threshold value is found exactly: one
 //            histogram of 1024 bins of 1/64 octave around 1/n locates its bin, the few
 //            entries of that bin are ranked against one another; a bin outside the window
-//            or with more than 64 entries falls back to three radix passes over all bits;
+//            or with more than 64 entries falls back to four 8-bit radix passes over all bits;
 //   step 2-3 hits: CRF <- lambda^(t - tau) CRF + 1, tau <- t; misses only get the decayed
 //            CRF_temp, which is not stored;
 //   step 4   the entries lowest under (CRF_temp, tau, position) leave until the head is
@@ -19,7 +19,7 @@
 
 namespace ckv {
 
-constexpr int HIST_BINS = 2048;
+constexpr int HIST_BINS = 1024;   // shared histogram size: the fine pass uses all of it, a radix pass 256
 constexpr float MASS_ONE = 1099511627776.0f;   // 2^40
 
 constexpr int FINE_BINS = 1024;   // fast path: bins of 2^17 key steps = 1/64 octave, 16 octaves wide
@@ -37,8 +37,38 @@ struct LrfuSmem {
   int ncand;
   int star;
   int eq[NW];
-  int amin[NW * 4];
+  int amin[NW * 5];
+  int last[4];   // slot, position, tau, CRF bits of list position n-1 after the update
   int ev[320];
+};
+
+// Loads the compiler must leave where they are written: the kernel is bound by the latency of
+// its dependent global reads (several microseconds each while the attention kernel saturates
+// HBM), so every read whose address is known is requested up front, in one batch.
+__device__ __forceinline__ int ld_i32(const int* p) {
+  int v;
+  asm volatile("ld.global.b32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ float ld_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.f32 %0, [%1];\n" : "=f"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ float4 ld_f32x4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+  return v;
+}
+
+constexpr int FRONT = 5;   // entries per thread whose logit rows are requested before n is known
+
+// What the kernel requests before it knows the head's length.
+template <int G>
+struct Front {
+  float4 ra[FRONT], rb[FRONT];   // logit rows of entries tid, tid + NT, ... (index clamped to the scratch)
+  float m[G], l[G];              // merged reference point (log2 domain) and normaliser per query head
+  int budget;
 };
 
 __device__ __forceinline__ unsigned long long mass_of(float pm) { return (unsigned long long)(pm * MASS_ONE); }
@@ -46,7 +76,7 @@ __device__ __forceinline__ unsigned long long mass_of(float pm) { return (unsign
 // EPT > 0: every thread keeps the pbar of its entries tid, tid + NT, ... (at most EPT) in
 // registers; EPT == 0: they live in the global scratch and any n is allowed.
 template <int G, int EPT>
-__device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n, LrfuSmem& sh) {
+__device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n, LrfuSmem& sh, const Front<G>& fr) {
   constexpr int R = EPT > 0 ? EPT : 1;
   const State& st = p.st;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -59,8 +89,8 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   float mx[G], invl[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
-    mx[g] = p.sc.mfin[u * (2 * QH) + g] * 0.693147180559945309f;   // log2 domain -> natural log
-    invl[g] = 1.0f / (p.sc.mfin[u * (2 * QH) + QH + g] * (float)G);
+    mx[g] = fr.m[g] * 0.693147180559945309f;   // log2 domain -> natural log
+    invl[g] = 1.0f / (fr.l[g] * (float)G);
   }
   auto pbar_of = [&](int i) {
     const float4 a = *reinterpret_cast<const float4*>(S + (size_t)i * QH);
@@ -73,23 +103,27 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     return pm;
   };
   float pmr[R];
-  if (EPT > 0 && EPT <= 8) {
-    // all logit rows first (clamped index, no branch), so that their latencies overlap
-    float4 ra[R], rb[R];
+  // stored state of this thread's entries, requested as soon as the logits are consumed so that
+  // the reads complete under the threshold search (EPT == FRONT only)
+  int pos_r[R], tau_r[R], slot_last = 0;
+  float crf_r[R];
+  if (EPT == FRONT) {
 #pragma unroll
     for (int k = 0; k < R; ++k) {
-      const int i = min(tid + k * NT, n - 1);
-      ra[k] = *reinterpret_cast<const float4*>(S + (size_t)i * QH);
-      rb[k] = (G > 4) ? *reinterpret_cast<const float4*>(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int k = 0; k < R; ++k) {
-      const float sv[8] = {ra[k].x, ra[k].y, ra[k].z, ra[k].w, rb[k].x, rb[k].y, rb[k].z, rb[k].w};
+      const float sv[8] = {fr.ra[k].x, fr.ra[k].y, fr.ra[k].z, fr.ra[k].w, fr.rb[k].x, fr.rb[k].y, fr.rb[k].z, fr.rb[k].w};
       float pm = 0.f;
 #pragma unroll
       for (int g = 0; g < G; ++g) pm = fmaf(expf(sv[g] - mx[g]), invl[g], pm);
       pmr[k] = (tid + k * NT < n) ? pm : 0.f;
     }
+#pragma unroll
+    for (int k = 0; k < R; ++k) {
+      const size_t i = mb + min(tid + k * NT, n - 1);
+      pos_r[k] = ld_i32(st.meta_pos + i);
+      tau_r[k] = ld_i32(st.meta_tau + i);
+      crf_r[k] = ld_f32(st.meta_crf + i);
+    }
+    if (tid == (n - 1) % NT) slot_last = ld_i32(st.list_slot + mb + n - 1);   // the owner of the last entry
   } else if (EPT > 0) {
 #pragma unroll
     for (int k = 0; k < R; ++k) {
@@ -212,13 +246,13 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     }
   }
   if (!found_all) {
-    // ---- general path: MSB-first radix passes over the fp32 bits of pbar (11, 11, 10 bits)
+    // ---- general path: MSB-first radix passes over the fp32 bits of pbar, 8 bits each
     A = 0;
     uint32_t prefix = 0;
     found_all = true;
-    for (int pass = 0; pass < 3; ++pass) {
-      const int sft = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-      const int wid = pass == 2 ? 10 : 11;
+    for (int pass = 0; pass < 4; ++pass) {
+      const int sft = 24 - 8 * pass;
+      const int wid = 8;
       const int nb = 1 << wid;
       __syncthreads();
       for (int b = tid; b < nb; b += NT) { sh.hist_lo[b] = 0u; sh.hist_hi[b] = 0u; }
@@ -308,7 +342,7 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   const unsigned long long w_theta = mass_of(__uint_as_float(theta));
 
   // ---- steps 2-3: CRF/tau update; step 4 candidates
-  const int k_evict = n - st.budget[uid];
+  const int k_evict = n - fr.budget;
   uint32_t bk0 = 0xffffffffu, bk1 = 0xffffffffu, bk2 = 0xffffffffu;
   int bidx = -1, nhit = 0;
   auto update = [&](int i, float pm, int pos_i, int tau, float crf, float dec) {
@@ -345,22 +379,23 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       }
     }
   } else if (EPT > 0) {
-    int pos_r[R], tau_r[R];
-    float crf_r[R], dec_r[R];
+    float dec_r[R];
 #pragma unroll
-    for (int k = 0; k < R; ++k) {   // all loads first: they overlap
-      const int i = tid + k * NT;
-      const bool ok = k < kmax && i < n;
-      pos_r[k] = ok ? st.meta_pos[mb + i] : 0;
-      tau_r[k] = ok ? st.meta_tau[mb + i] : p.t;
-      crf_r[k] = ok ? st.meta_crf[mb + i] : 0.f;
-    }
-#pragma unroll
-    for (int k = 0; k < R; ++k) dec_r[k] = __ldg(st.tab + (p.t - tau_r[k]));
+    for (int k = 0; k < R; ++k) dec_r[k] = __ldg(st.tab + (p.t - min(tau_r[k], p.t)));
 #pragma unroll
     for (int k = 0; k < R; ++k) {
       const int i = tid + k * NT;
-      if (k < kmax && i < n) update(i, pmr[k], pos_r[k], tau_r[k], crf_r[k], dec_r[k]);
+      if (i < n) {
+        const int nh = nhit;
+        update(i, pmr[k], pos_r[k], tau_r[k], crf_r[k], dec_r[k]);
+        if (i == n - 1) {   // what list position n-1 holds after this step, for the in-place swap
+          const bool hit = nhit != nh;
+          sh.last[0] = slot_last;
+          sh.last[1] = pos_r[k];
+          sh.last[2] = hit ? p.t : tau_r[k];
+          sh.last[3] = __float_as_int(hit ? __fadd_rn(__fmul_rn(dec_r[k], crf_r[k]), 1.0f) : crf_r[k]);
+        }
+      }
     }
   } else {
     for (int i = tid; i < n; i += NT) {
@@ -372,27 +407,39 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   if (lane == 0 && nhit) atomicAdd(&st.counters[1], (unsigned long long)nhit);
   int n_after = n;
   if (k_evict == 1) {
-    // block argmin of (CRF_temp, tau, pos)
+    // block argmin of (CRF_temp, tau, pos); every thread asks for the slot of its own candidate
+    // now, so the winner's is at hand when the reduction ends
+    int bslot = (EPT == FRONT && bidx >= 0) ? ld_i32(st.list_slot + mb + bidx) : 0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const uint32_t o0 = __shfl_xor_sync(0xffffffffu, bk0, o), o1 = __shfl_xor_sync(0xffffffffu, bk1, o),
                      o2 = __shfl_xor_sync(0xffffffffu, bk2, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bidx, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bidx, o), os = __shfl_xor_sync(0xffffffffu, bslot, o);
       const bool less = (o0 != bk0) ? (o0 < bk0) : ((o1 != bk1) ? (o1 < bk1) : (o2 < bk2));
-      if (less) { bk0 = o0; bk1 = o1; bk2 = o2; bidx = oi; }
+      if (less) { bk0 = o0; bk1 = o1; bk2 = o2; bidx = oi; bslot = os; }
     }
-    if (lane == 0) { sh.amin[w * 4] = (int)bk0; sh.amin[w * 4 + 1] = (int)bk1; sh.amin[w * 4 + 2] = (int)bk2; sh.amin[w * 4 + 3] = bidx; }
+    if (lane == 0) { sh.amin[w * 5] = (int)bk0; sh.amin[w * 5 + 1] = (int)bk1; sh.amin[w * 5 + 2] = (int)bk2; sh.amin[w * 5 + 3] = bidx; sh.amin[w * 5 + 4] = bslot; }
     __syncthreads();   // also orders every CRF/tau store above before the swap below
     if (tid == 0) {
       uint32_t a0 = (uint32_t)sh.amin[0], a1 = (uint32_t)sh.amin[1], a2 = (uint32_t)sh.amin[2];
-      int ai = sh.amin[3];
+      int ai = sh.amin[3], as = sh.amin[4];
       for (int x = 1; x < NW; ++x) {
-        const uint32_t o0 = (uint32_t)sh.amin[x * 4], o1 = (uint32_t)sh.amin[x * 4 + 1], o2 = (uint32_t)sh.amin[x * 4 + 2];
+        const uint32_t o0 = (uint32_t)sh.amin[x * 5], o1 = (uint32_t)sh.amin[x * 5 + 1], o2 = (uint32_t)sh.amin[x * 5 + 2];
         const bool less = (o0 != a0) ? (o0 < a0) : ((o1 != a1) ? (o1 < a1) : (o2 < a2));
-        if (less) { a0 = o0; a1 = o1; a2 = o2; ai = sh.amin[x * 4 + 3]; }
+        if (less) { a0 = o0; a1 = o1; a2 = o2; ai = sh.amin[x * 5 + 3]; as = sh.amin[x * 5 + 4]; }
       }
       // the leaving entry's slot becomes the head's spare at position n-1
-      if (ai != n - 1) swap_into(st, mb, ai, n - 1);
+      if (ai != n - 1) {
+        if (EPT == FRONT) {   // everything needed is already here: stores only
+          st.list_slot[mb + ai] = sh.last[0];
+          st.meta_pos[mb + ai] = sh.last[1];
+          st.meta_tau[mb + ai] = sh.last[2];
+          st.meta_crf[mb + ai] = __int_as_float(sh.last[3]);
+          st.list_slot[mb + n - 1] = as;
+        } else {
+          swap_into(st, mb, ai, n - 1);
+        }
+      }
       p.n_out[uid] = n - 1;
       atomicAdd(&st.counters[2], 1ull);
     }
@@ -413,14 +460,33 @@ __global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
   const State& st = p.st;
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
   const int uid = (seq * st.L + p.layer) * st.H + head;
-  const int n = p.n_in[uid] + p.append;
+  // one batch of requests: the length, the budget, the softmax reference, and the logit rows the
+  // common path needs (requested for a full thread's worth, clamped to the scratch)
+  const int n_raw = ld_i32(p.n_in + uid);
+  Front<G> fr;
+  fr.budget = ld_i32(st.budget + uid);
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    fr.m[g] = ld_f32(p.sc.mfin + u * (2 * QH) + g);
+    fr.l[g] = ld_f32(p.sc.mfin + u * (2 * QH) + QH + g);
+  }
+  {
+    const float* S = p.sc.logits + (size_t)u * p.sc.cap_s * QH;
+#pragma unroll
+    for (int k = 0; k < FRONT; ++k) {
+      const int i = min((int)threadIdx.x + k * NT, p.sc.cap_s - 1);
+      fr.ra[k] = ld_f32x4(S + (size_t)i * QH);
+      fr.rb[k] = (G > 4) ? ld_f32x4(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  const int n = n_raw + p.append;
   if (n <= 0) {
     if (threadIdx.x == 0) p.n_out[uid] = 0;
     return;
   }
-  if (n <= 5 * NT) lrfu_unit<G, 5>(p, u, uid, seq, n, sh);
-  else if (n <= 17 * NT) lrfu_unit<G, 17>(p, u, uid, seq, n, sh);
-  else lrfu_unit<G, 0>(p, u, uid, seq, n, sh);
+  if (n <= FRONT * NT) lrfu_unit<G, FRONT>(p, u, uid, seq, n, sh, fr);
+  else if (n <= 17 * NT) lrfu_unit<G, 17>(p, u, uid, seq, n, sh, fr);
+  else lrfu_unit<G, 0>(p, u, uid, seq, n, sh, fr);
 }
 
 }  // namespace ckv
