@@ -71,6 +71,26 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// The same with an L2 eviction policy for the lines it touches.
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
+// Cache rows are read once per step and the whole cache is far larger than L2: they should
+// leave L2 first.  The step's logits are read back by the LRFU kernel a little later: last.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void st_f32x2_hint(float* p, float a, float b, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;\n" ::"l"(p), "f"(a), "f"(b), "l"(pol) : "memory");
+}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
@@ -222,6 +242,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   const uint32_t kb = (uint32_t)(((mi & 1) * 8 + r8) * ENTRY_STRIDE + (mi >> 1) * 16);
   const uint32_t vb = (uint32_t)(ROW_BYTES + ((mi >> 1) * 8 + r8) * ENTRY_STRIDE + (mi & 1) * 16);
 
+  const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
   int fsi = 0, csi = 0;     // stage the next fire fills / the next compute reads
   uint32_t phases = 0;      // bit s: parity of the next completion of stage s
   bool waited = p.early == 0;
@@ -259,7 +280,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
       const int nv = valid - has_new;                   // entries that come from the pool
       if (lane == 0) mbar_expect_tx(bar, (uint32_t)valid * SLOT_BYTES);
       __syncwarp();
-      if (lane < nv) bulk_g2s(stage + lane * ENTRY_STRIDE, pool + (size_t)(unsigned)slot * SLOT_BYTES, SLOT_BYTES, bar);
+      if (lane < nv) bulk_g2s_hint(stage + lane * ENTRY_STRIDE, pool + (size_t)(unsigned)slot * SLOT_BYTES, SLOT_BYTES, bar, pol_stream);
       if (has_new) {   // it comes from the call's inputs
         if (!waited) { pdl_wait(); waited = true; }
         if (lane < 2)
@@ -358,8 +379,8 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
       const bool v0 = gid < valid, v1 = gid + 8 < valid;
       if (p.track) {
         float* lrow = lrow0 + (size_t)base * QH;
-        if (v0) *reinterpret_cast<float2*>(lrow) = make_float2(__fmul_rn(s[0], p.scale), __fmul_rn(s[1], p.scale));
-        if (v1) *reinterpret_cast<float2*>(lrow + 8 * QH) = make_float2(__fmul_rn(s[2], p.scale), __fmul_rn(s[3], p.scale));
+        if (v0) st_f32x2_hint(lrow, __fmul_rn(s[0], p.scale), __fmul_rn(s[1], p.scale), pol_keep);
+        if (v1) st_f32x2_hint(lrow + 8 * QH, __fmul_rn(s[2], p.scale), __fmul_rn(s[3], p.scale), pol_keep);
       }
       // ---- online softmax, this lane's two heads (2 tig, 2 tig + 1) over its two keys
       const float t0 = v0 ? s[0] * p.scale_log2 : -INFINITY, t1 = v0 ? s[1] * p.scale_log2 : -INFINITY;
