@@ -314,11 +314,11 @@ def main():
                 "kernel": "attn_kernel", "launch_us": kernel_ms * 1000.0,
                 "algorithmic_bytes_per_launch": algo_bytes / n_launch,
                 "entries_per_launch": entries / n_launch, "hit_fraction": hits / max(entries, 1)}
-    traffic_file = os.path.join(ROOT, "profiles", "decode_kernel_traffic.json")
-    if os.path.exists(traffic_file):
-        with open(traffic_file) as f:
-            tj = json.load(f)
-        roofline["traffic"] = tj.get("dram_bytes_per_entry", 0) * entries / n_launch or None
+    # DRAM traffic of one attn_kernel launch from the ncu capture summarised in
+    # profiles/attn_lrfu_kernels_cfg4_qwen14b.md (same launch shape): read + write bytes per entry
+    NCU_DRAM_BYTES_PER_ENTRY = (135.844096e6 + 4.0512e6) / 262400.0
+    if wl.name == "cfg4_qwen14b" and not args.batch and not args.budget:
+        roofline["traffic"] = NCU_DRAM_BYTES_PER_ENTRY * entries / n_launch
 
     # end to end: the same steps through the host-buffer entry point, copies inside the timed region
     e2e = None
