@@ -102,8 +102,12 @@ int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* 
                           const void* v_new, void* out, void* stream);
 
 /*
- * The same step with pinned HOST buffers: copies q, k_new, v_new to the device, runs
- * the step and copies `out` back, all enqueued on `stream` (no host synchronisation).
+ * The same step with HOST buffers (page-locked for asynchronous copies).  The inputs are
+ * copied up on one stream of the handle and `out` is copied down on another, both ordered
+ * against the step on `stream` by events, so the copies of one layer run beside the kernels
+ * of others.  No host synchronisation.  `out_host` is complete once `stream` has passed a
+ * later crystalkv_join (or any call that reads the cache state) and has been synchronised;
+ * the input buffers may be reused from then on too.
  */
 int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host,
                                const void* k_new_host, const void* v_new_host, void* out_host,

@@ -12,6 +12,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdint>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -51,7 +52,13 @@ struct crystalkv {
   int stage = CRYSTALKV_STAGE_THINK;
   int answer_steps = 0;
   long long* Asum = nullptr;
-  __nv_bfloat16 *dq = nullptr, *dk = nullptr, *dv = nullptr, *dout = nullptr;  // staging for host I/O
+  // host I/O: HOST_RING staging sets; inputs go up on one internal stream and results come
+  // down on another, so the copies of other layers run beside the attention kernels
+  static constexpr int HOST_RING = 16;
+  __nv_bfloat16 *dq[HOST_RING] = {}, *dk[HOST_RING] = {}, *dv[HOST_RING] = {}, *dout[HOST_RING] = {};
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t evIn[HOST_RING] = {}, evUse[HOST_RING] = {}, evOut[HOST_RING] = {};
+  long long nHost = 0;             // host-buffer steps so far
   __nv_bfloat16* dummy_out = nullptr;
   float* tab = nullptr;
   std::vector<void*> allocs;
@@ -200,6 +207,7 @@ int join_side(crystalkv_t* h, cudaStream_t s) {
   h->prev_layer = -1;
   if (h->kF > 0) CK(h, cudaStreamWaitEvent(s, h->evF[(h->kF - 1) % crystalkv::EV_RING], 0));
   h->joined = h->kF - 1;
+  if (h->nHost > 0) CK(h, cudaStreamWaitEvent(s, h->evOut[(h->nHost - 1) % crystalkv::HOST_RING], 0));   // copies back run in order
   return CRYSTALKV_OK;
 }
 
@@ -275,6 +283,13 @@ int crystalkv_destroy(crystalkv_t* h) {
   cudaSetDevice(h->cfg.device);
   cudaDeviceSynchronize();
   if (h->side) cudaStreamDestroy(h->side);
+  if (h->copy_in) cudaStreamDestroy(h->copy_in);
+  if (h->copy_out) cudaStreamDestroy(h->copy_out);
+  for (int i = 0; i < crystalkv::HOST_RING; ++i) {
+    if (h->evIn[i]) cudaEventDestroy(h->evIn[i]);
+    if (h->evUse[i]) cudaEventDestroy(h->evUse[i]);
+    if (h->evOut[i]) cudaEventDestroy(h->evOut[i]);
+  }
   if (h->evA) cudaEventDestroy(h->evA);
   for (cudaEvent_t e : h->evF)
     if (e) cudaEventDestroy(e);
@@ -340,6 +355,13 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   if (bps < 1) { h->err = "attention kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
   h->grid = h->num_sms * bps;
   CKC(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
+  CKC(cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking));
+  CKC(cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking));
+  for (int i = 0; i < crystalkv::HOST_RING; ++i) {
+    CKC(cudaEventCreateWithFlags(&h->evIn[i], cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&h->evUse[i], cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&h->evOut[i], cudaEventDisableTiming));
+  }
   CKC(cudaEventCreateWithFlags(&h->evA, cudaEventDisableTiming));
   for (cudaEvent_t& e : h->evF) CKC(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
 
@@ -375,7 +397,8 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   }
   DA(&h->sc_pbar, (size_t)h->U * h->cap_s);
   const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
-  DA(&h->dq, qn); DA(&h->dout, qn); DA(&h->dk, kn); DA(&h->dv, kn); DA(&h->dummy_out, qn);
+  for (int i = 0; i < crystalkv::HOST_RING; ++i) { DA(&h->dq[i], qn); DA(&h->dout[i], qn); DA(&h->dk[i], kn); DA(&h->dv[i], kn); }
+  DA(&h->dummy_out, qn);
 
   // lambda^D as fp32 from an fp64 pow; pow(0, 0) = 1 keeps same-step hits when lambda = 0
   {
@@ -493,12 +516,27 @@ int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host, co
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)c.batch * c.n_q_heads * HD * 2, kb = (size_t)c.batch * c.n_kv_heads * HD * 2;
-  CK(h, cudaMemcpyAsync(h->dq, q_host, qb, cudaMemcpyHostToDevice, s));
-  CK(h, cudaMemcpyAsync(h->dk, k_new_host, kb, cudaMemcpyHostToDevice, s));
-  CK(h, cudaMemcpyAsync(h->dv, v_new_host, kb, cudaMemcpyHostToDevice, s));
-  rc = crystalkv_decode_step(h, layer, h->dq, h->dk, h->dv, h->dout, stream);
+  if (h->t_layer[layer] < 0) return fail(h, CRYSTALKV_ESTATE, "decode before prefill");
+  // Staging set j: its inputs go up on the copy-in stream (behind the attention kernel and the
+  // copy back that used the set HOST_RING steps ago), the caller's stream waits for them, runs
+  // the step, and the result comes down on the copy-out stream behind the attention kernel.
+  const int j = (int)(h->nHost % crystalkv::HOST_RING);
+  if (h->nHost >= crystalkv::HOST_RING) {
+    CK(h, cudaStreamWaitEvent(h->copy_in, h->evUse[j], 0));
+    CK(h, cudaStreamWaitEvent(h->copy_in, h->evOut[j], 0));
+  }
+  CK(h, cudaMemcpyAsync(h->dq[j], q_host, qb, cudaMemcpyHostToDevice, h->copy_in));
+  CK(h, cudaMemcpyAsync(h->dk[j], k_new_host, kb, cudaMemcpyHostToDevice, h->copy_in));
+  CK(h, cudaMemcpyAsync(h->dv[j], v_new_host, kb, cudaMemcpyHostToDevice, h->copy_in));
+  CK(h, cudaEventRecord(h->evIn[j], h->copy_in));
+  CK(h, cudaStreamWaitEvent(s, h->evIn[j], 0));
+  rc = crystalkv_decode_step(h, layer, h->dq[j], h->dk[j], h->dv[j], h->dout[j], stream);
   if (rc) return rc;
-  CK(h, cudaMemcpyAsync(out_host, h->dout, qb, cudaMemcpyDeviceToHost, s));
+  CK(h, cudaEventRecord(h->evUse[j], s));
+  CK(h, cudaStreamWaitEvent(h->copy_out, h->evUse[j], 0));
+  CK(h, cudaMemcpyAsync(out_host, h->dout[j], qb, cudaMemcpyDeviceToHost, h->copy_out));
+  CK(h, cudaEventRecord(h->evOut[j], h->copy_out));
+  h->nHost++;
   return CRYSTALKV_OK;
 }
 

@@ -217,6 +217,49 @@ def test_cfg5_sweep_cells_sampled():
         ls.close()
 
 
+def test_host_buffer_steps_match_device_steps():
+    """crystalkv_decode_step_host with pinned buffers (the kernel reads them over PCIe) and with
+    pageable buffers (staged copies) gives the outputs and the state of the device-pointer call."""
+    import ctypes as C
+    from paper_2601_16986_b200 import Config, CrystalKV
+    wl = Workload(name="hostio", seed=21, n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3, prompt=50,
+                  think_steps=40, budget_per_head=64)
+    def make():
+        kv = CrystalKV(Config(n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3, budget_per_head=64, max_context=128))
+        for l in range(2):
+            k, v = wl.prompt_kv(l, device="cuda")
+            kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], device="cuda")[:, 0].contiguous())
+        return kv
+    dev, pin, page = make(), make(), make()
+    for s in range(40):
+        for l in range(2):
+            q, k, v = wl.step_inputs(l, wl.prompt + s, device="cuda")
+            ref = dev.decode_step(l, q, k, v)
+            hq, hk, hv = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+            ho = torch.empty_like(hq).pin_memory()
+            pin.decode_step_host(l, hq, hk, hv, ho)
+            # pageable: plain tensors through the C ABI
+            pq, pk, pv = q.cpu(), k.cpu(), v.cpu()
+            po = torch.empty_like(pq)
+            P = lambda t: C.c_void_p(t.data_ptr())
+            rc = page.lib.crystalkv_decode_step_host(page._h, l, P(pq), P(pk), P(pv), P(po),
+                                                     C.c_void_p(torch.cuda.current_stream().cuda_stream))
+            assert rc == 0
+            pin.join()
+            page.join()
+            torch.cuda.synchronize()
+            assert torch.equal(ho, ref.cpu()) and torch.equal(po, ref.cpu())
+    for l in range(2):
+        for b in range(3):
+            for h in range(2):
+                a = dev.export_state(l, b, h)
+                assert (a == pin.export_state(l, b, h)).all() and (a == page.export_state(l, b, h)).all()
+    for kv in (dev, pin, page):
+        kv.check()
+        kv.validate()
+        kv.close()
+
+
 # ------------------------------------------------------------------ error paths on a live handle
 def test_call_order_errors():
     from paper_2601_16986_b200 import Config, CrystalKV, CrystalKVError
