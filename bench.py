@@ -176,6 +176,95 @@ def run_reference(args, wl):
 
 
 # ---------------------------------------------------------------------------------------
+def sweep_cell(wl, batch, budget, fullkv, context, steps, warmup, dev):
+    """Steady-state decode of the 14B shape at one (batch, budget) cell, or of the full-cache
+    baseline with `context` entries per head; returns a dict for one table row."""
+    from paper_2601_16986_b200 import Config, CrystalKV, CrystalKVError, FULLKV, EVICT
+    L, Hq, H, d = wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    P = context - 1 if fullkv else budget
+    total = warmup + steps
+    row = {"batch": batch, "budget": None if fullkv else budget, "mode": "fullkv" if fullkv else "crystal-kv",
+           "entries_per_head": context if fullkv else budget + 1}
+    need_gb = batch * L * H * (P + total + 2) * 512 / 1e9
+    if need_gb > 150:
+        row["status"] = f"OOM: {need_gb:.0f} GB of K/V rows"
+        return row
+    try:
+        kv = CrystalKV(Config(n_layers=L, n_q_heads=Hq, n_kv_heads=H, batch=batch, budget_per_head=budget,
+                              max_context=P + total + 2, mode=FULLKV if fullkv else EVICT, top_p=wl.top_p, lam=wl.lam))
+    except CrystalKVError as e:
+        row["status"] = f"create failed: {e}"
+        return row
+    w = wl.scaled(batch=batch, prompt=P)
+    with torch.no_grad():
+        if fullkv:   # values do not matter for the baseline's timing: one prompt tensor serves every layer
+            k, v = w.prompt_kv(0, device=dev)
+            q = w.queries(0, [P - 1], device=dev)[:, 0].contiguous()
+            for l in range(L):
+                kv.prefill(l, k, v, q)
+            del k, v
+        else:
+            for l in range(L):
+                k, v = w.prompt_kv(l, device=dev)
+                kv.prefill(l, k, v, w.queries(l, [P - 1], device=dev)[:, 0].contiguous())
+                del k, v
+        NS = total   # every step its own inputs: repeated keys would put exact ties into the cache
+        pos = torch.arange(P, P + NS)
+        lay = range(L) if not fullkv else [0] * L
+        Q = torch.stack([w.queries(l, pos, device=dev).transpose(0, 1) for l in lay], 1).contiguous()
+        K = torch.stack([w.keys(l, pos, device=dev).transpose(0, 1) for l in lay], 1).contiguous()
+        V = torch.stack([w.values(l, pos, device=dev).transpose(0, 1) for l in lay], 1).contiguous()
+        OUT = torch.empty(L, batch, Hq, d, dtype=torch.bfloat16, device=dev)
+    lib, h = kv.lib, kv._h
+    stream = torch.cuda.current_stream()
+    sp = C.c_void_p(stream.cuda_stream)
+    P_ = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
+
+    def run(n0, n1):
+        for s in range(n0, n1):
+            i = s % NS
+            for l in range(L):
+                rc = lib.crystalkv_decode_step(h, l, P_(Q[i, l]), P_(K[i, l]), P_(V[i, l]), P_(OUT[l]), sp)
+                if rc:
+                    raise RuntimeError(f"decode_step failed: {rc}")
+    run(0, warmup)
+    torch.cuda.synchronize()
+    c0 = kv.get_counters()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    run(warmup, total)
+    lib.crystalkv_join(h, sp)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    c1 = kv.get_counters()
+    kv.check()
+    entries = (c1["entries_attended"] - c0["entries_attended"]) / steps
+    peak, _ = measured_peaks()
+    gbs = entries * 512 / (ms / 1000.0) / 1e9
+    row.update({"status": "ok", "ms_per_step": ms, "steps_per_s": 1000.0 / ms, "kv_gb_per_step": entries * 512 / 1e9,
+                "kv_gb_per_s": gbs, "frac_of_measured_hbm": gbs / peak})
+    kv.close()
+    del Q, K, V, OUT
+    torch.cuda.empty_cache()
+    return row
+
+
+def run_sweep(args):
+    """The 14B-shape sweep: batch x per-head budget in steady state, and the full-cache baseline
+    (every one of `context` tokens kept) of the same library; one JSON line per cell."""
+    wl = WORKLOADS["cfg5_sweep14b"]
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    context = args.context
+    for batch in (1, 8, 32, 128):
+        row = sweep_cell(wl, batch, 1024, True, context, 8, 3, dev)
+        print(json.dumps(row), flush=True)
+        for budget in (256, 1024, 4096):
+            row = sweep_cell(wl, batch, budget, False, context, args.steps, max(args.warmup, 3), dev)
+            print(json.dumps(row), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -188,6 +277,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")
     ap.add_argument("--e2e-steps", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="14B-shape sweep (batch x budget, steady state) against the full-cache baseline; one JSON line per cell")
+    ap.add_argument("--context", type=int, default=32768, help="tokens kept per head by the full-cache baseline of --sweep")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     if args.batch:
@@ -198,6 +290,10 @@ def main():
         wl = wl.scaled(n_layers=args.layers)
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.sweep:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        return run_sweep(args)
     if args.warmup < 3:
         raise SystemExit("--warmup must be at least 3")
 
