@@ -109,6 +109,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
   }
 }
 
+constexpr int PIECE_SOFT = 24;  // groups a piece may grow to when that saves merge rounds
 constexpr float LAZY = 8.0f;   // the running maximum (log2 domain) may trail the true one by this much
 
 // Accumulates HB heads x PB pieces of split-K partials for 4 output channels per lane; every
@@ -190,6 +191,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   int* off = reinterpret_cast<int*>(smem + RING_BYTES + NW * STAGES * 8);   // U + 1 piece prefix sums
   int* nin = off + (U + 1);                                                  // U entry counts before the step
   __shared__ int s_red[NW + 1];
+  __shared__ int s_mx[NW];
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
   const int G = p.G;
   const int PS = 16 + G * HD;
@@ -201,17 +203,26 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   const int nWarps = gridDim.x * NW;
   int T;
   {
-    int mine = 0;
+    int mine = 0, gmax = 0;
     for (int u = tid; u < U; u += NT) {
       const int uid = ((u / st.H) * st.L + p.layer) * st.H + (u % st.H);
       const int n = p.n_in[uid];
       nin[u] = n;
-      mine += (n + p.append + GRP - 1) / GRP;
+      const int g = (n + p.append + GRP - 1) / GRP;
+      mine += g;
+      gmax = max(gmax, g);
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
+    if (lane == 0) s_mx[w] = gmax;
     int Gtot;
-    block_excl_scan(mine, s_red, Gtot);
+    block_excl_scan(mine, s_red, Gtot);   // its barriers also publish s_mx
     if (Gtot == 0) return;
+    for (int x = 0; x < NW; ++x) gmax = max(gmax, s_mx[x]);
     T = (nWarps > U) ? (Gtot + (nWarps - U) - 1) / (nWarps - U) : 0x7fffffff;
+    // Small launches have warps to spare: pieces of up to PIECE_SOFT groups keep a unit at four
+    // pieces or fewer, which the merge handles in a single round of loads.
+    T = max(T, min(PIECE_SOFT, (gmax + 3) / 4));
     T = max(T, GMIN);
     int run = 0;
     for (int b0 = 0; b0 < U; b0 += NT) {
@@ -230,8 +241,25 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
     __syncthreads();
   }
   const int Ptot = off[U];
-  const int me = w * gridDim.x + blockIdx.x;   // ranks interleave over the CTAs so small launches use every SM
-  if (me >= Ptot) return;
+  // Which piece a warp takes.  When every warp gets at most one, pieces go to the warps in the
+  // order in which they become ready (one atomic each): CTAs that reach an SM late, because the
+  // kernel ahead held it longer, then find the pieces gone instead of finishing last.  The
+  // counter of the other parity is cleared for the next launch: all takes of the launch before
+  // this one happened before it let this one start.
+  const bool dyn = Ptot <= nWarps;
+  if (blockIdx.x == 0 && tid == 0) {
+    atomicExch(p.piece_ctr + (p.parity ^ 1), 0);
+    __threadfence();
+  }
+  int pi;
+  if (dyn) {
+    pi = 0;
+    if (lane == 0) pi = atomicAdd(p.piece_ctr + p.parity, 1);
+    pi = __shfl_sync(0xffffffffu, pi, 0);
+  } else {
+    pi = w * gridDim.x + blockIdx.x;   // ranks interleave over the CTAs
+  }
+  if (pi >= Ptot) return;
 
   const uint32_t ring_u32 = smem_u32(smem) + w * (STAGES * STAGE_BYTES);
   const int gid = lane >> 2, tig = lane & 3;
@@ -248,7 +276,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   bool waited = p.early == 0;
 
 #pragma unroll 1
-  for (int pi = me; pi < Ptot; pi += nWarps) {
+  for (; pi < Ptot; pi += (dyn ? Ptot : nWarps)) {
     // ---- the piece: head u, groups [lo, hi) of its list
     int u;
     {

@@ -39,6 +39,7 @@ struct crystalkv {
   float* sc_partials[2] = {};
   int* sc_ticket[2] = {};
   float* sc_pbar = nullptr;
+  int* piece_ctr = nullptr;
   int cap_s = 0, pmax = 0;
   long long nA = 0;                // attention launches so far
   std::vector<int> t_layer, par;   // per layer: time of the last step, current count buffer
@@ -187,6 +188,8 @@ DecodeParams make_params(crystalkv_t* h, int layer, int set) {
   p.sc.cap_s = h->cap_s;
   p.sc.pmax = h->pmax;
   p.sc.pbar = h->sc_pbar;
+  p.piece_ctr = h->piece_ctr;
+  p.parity = (int)(h->nA & 1);
   p.sc.partials = h->sc_partials[h->nA & 1];
   p.sc.ticket = h->sc_ticket[h->nA & 1];
   p.sc.logits = h->sc_logits[0];
@@ -396,6 +399,8 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     CKC(cudaMemset(h->sc_ticket[i], 0, (size_t)h->U * sizeof(int)));
   }
   DA(&h->sc_pbar, (size_t)h->U * h->cap_s);
+  DA(&h->piece_ctr, 2);
+  CKC(cudaMemset(h->piece_ctr, 0, 2 * sizeof(int)));
   const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
   for (int i = 0; i < crystalkv::HOST_RING; ++i) { DA(&h->dq[i], qn); DA(&h->dout[i], qn); DA(&h->dk[i], kn); DA(&h->dv[i], kn); }
   DA(&h->dummy_out, qn);
