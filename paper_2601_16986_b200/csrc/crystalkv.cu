@@ -387,7 +387,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   DA(&st.counters, 4);
   DA(&h->Asum, h->units);
   const int capgroups = (h->cap + GRP - 1) / GRP;
-  h->cap_s = evict ? h->cap : 1;
+  h->cap_s = evict ? ((h->cap + 3) & ~3) : 4;   // whole 128-byte lines of logit rows per unit
   h->pmax = capgroups / GMIN + 2;
   for (int i = 0; i < NSETS; ++i) {
     DA(&h->sc_logits[i], (size_t)h->U * h->cap_s * QH);

@@ -124,6 +124,23 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       crf_r[k] = ld_f32(st.meta_crf + i);
     }
     if (tid == (n - 1) % NT) slot_last = ld_i32(st.list_slot + mb + n - 1);   // the owner of the last entry
+    // The logit rows are dead now (every thread holds its own in registers since before the
+    // kernel learnt n, and nothing reads them again): drop their L2 lines instead of letting
+    // them be written back to DRAM later.  Four 32-byte rows share a 128-byte line; units start
+    // on line boundaries (cap_s is a multiple of four).
+    // The barrier takes a value computed from every pbar, so no thread passes it with a row
+    // load still in flight.
+    int unordered = 0;
+#pragma unroll
+    for (int k = 0; k < R; ++k) unordered |= (pmr[k] != pmr[k]);
+    (void)__syncthreads_or(unordered);
+    if ((tid & 3) == 0) {
+#pragma unroll
+      for (int k = 0; k < R; ++k) {
+        const int i = tid + k * NT;
+        if (i < n) asm volatile("discard.global.L2 [%0], 128;\n" ::"l"(S + (size_t)i * QH) : "memory");
+      }
+    }
   } else if (EPT > 0) {
 #pragma unroll
     for (int k = 0; k < R; ++k) {
