@@ -217,6 +217,39 @@ def test_cfg5_sweep_cells_sampled():
         ls.close()
 
 
+def test_more_heads_than_warps_in_the_grid():
+    """batch x kv heads above the attention grid's warp count (148 SMs x 8): every warp takes
+    several whole heads in turn instead of one piece."""
+    wl = Workload(name="wide", seed=61, n_layers=1, n_q_heads=24, n_kv_heads=8, batch=180, prompt=37,
+                  think_steps=24, budget_per_head=44, outlier="flat", outlier_frac=0.05)
+    ls = LockStep(wl, [0, 97, 179])
+    ls.prefill()
+    ls.compare()
+    for s in range(wl.think_steps):
+        ls.step(compare_state=(s % 4 == 3))
+    ls.compare()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert len(ls.gpu.get_retained(0, 179, 7)) == 44
+    ls.close()
+
+
+def test_very_long_heads_use_the_general_lrfu_path():
+    """A head above 17 x 256 entries: the LRFU kernel keeps pbar in global scratch, the attention
+    kernel cuts the head into many pieces (merge in several rounds)."""
+    wl = Workload(name="long", seed=62, n_layers=1, n_q_heads=4, n_kv_heads=1, batch=2, prompt=4500,
+                  think_steps=12, budget_per_head=4504)
+    ls = LockStep(wl, [0, 1])
+    ls.prefill()
+    ls.compare()
+    for s in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert len(ls.gpu.get_retained(0, 1, 0)) == 4504
+    ls.close()
+
+
 def test_host_buffer_steps_match_device_steps():
     """crystalkv_decode_step_host with pinned buffers (the kernel reads them over PCIe) and with
     pageable buffers (staged copies) gives the outputs and the state of the device-pointer call."""
