@@ -135,6 +135,15 @@ def oracle_sample(wl, layers: int, steps: int):
     return 1.0 / per_full_step, threads, desc
 
 
+def config_of(wl, world):
+    """The `config` object of the JSON line, the same for both arms."""
+    return {"workload": wl.name, "batch_per_gpu": wl.batch, "layers": wl.n_layers, "q_heads": wl.n_q_heads,
+            "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "budget_per_head": wl.budget_per_head,
+            "prompt": wl.prompt, "rebudget_every": wl.rebudget_every, "top_p": wl.top_p, "lambda": wl.lam,
+            "l2": "per-step working set (cache of all layers) far larger than L2; no flush",
+            "parallelism": f"replicas x{world}, no collective"}
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -168,8 +177,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.batch, "layers": wl.n_layers,
-                   "budget_per_head": wl.budget_per_head},
+        "config": config_of(wl, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -455,11 +463,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "batch_per_gpu": B, "layers": L, "q_heads": Hq, "kv_heads": H,
-                       "head_dim": d, "budget_per_head": wl.budget_per_head, "prompt": wl.prompt,
-                       "rebudget_every": every, "top_p": wl.top_p, "lambda": wl.lam,
-                       "l2": "per-step working set (cache of all layers) far larger than L2; no flush",
-                       "parallelism": f"replicas x{world}, no collective"},
+            "config": config_of(wl, world),
             "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches["n"],
             "roofline": roofline, "cpu_baseline": cpu,
             "rebudget_ms_in_timed_region": ms_rb,
