@@ -474,17 +474,18 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
         if (h1 < G) { po[h1 * HD + 16 * mt] = o[mt][1]; po[h1 * HD + 16 * mt + 8] = o[mt][3]; }
       }
     }
-    __threadfence();
+    // Release / acquire on the ticket: the warp barrier makes every lane's stores happen before
+    // lane 0's atomic, whose release makes them visible to the warp that acquires the last ticket.
     __syncwarp();
     int last = 0;
     if (lane == 0) {
-      const int old = atomicAdd(&p.sc.ticket[u], 1);
+      int old;
+      asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(p.sc.ticket + u) : "memory");
       last = (old == npieces - 1);
       if (last) p.sc.ticket[u] = 0;   // ready for the next launch that uses this scratch set
     }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) continue;
-    __threadfence();
     // ---- merge: out = sum_p O_p 2^(m_p - m) / sum_p l_p 2^(m_p - m).  The merging warp is alone,
     // so its time is the number of dependent load rounds: loads go out in batches before anything
     // consumes them.

@@ -18,7 +18,7 @@ constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;  // 198 KB
 constexpr int GMIN = 4;             // fewest groups a working warp takes
 constexpr int QH = 8;               // query heads of a group as padded for the MMA N dimension
 constexpr int MAX_UNITS_PER_CALL = 2048;   // bounded by the split tables in shared memory
-constexpr int NSETS = 8;            // logit scratch sets cycled by consecutive tracked launches
+constexpr int NSETS = 16;           // logit scratch sets cycled by consecutive tracked launches
 
 // error word bits raised by device-side consistency checks (never a trap)
 constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence's free list was empty

@@ -44,7 +44,7 @@ struct crystalkv {
   long long nA = 0;                // attention launches so far
   std::vector<int> t_layer, par;   // per layer: time of the last step, current count buffer
   // LRFU launches are numbered; launch k uses scratch set k % NSETS and event k % EV_RING
-  static constexpr int EV_RING = 16;
+  static constexpr int EV_RING = 32;
   cudaStream_t side = nullptr;
   cudaEvent_t evA = nullptr, evF[EV_RING] = {};
   long long kF = 0, joined = -1;
