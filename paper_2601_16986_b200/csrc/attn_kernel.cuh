@@ -109,6 +109,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
   }
 }
 
+constexpr int MAX_STAGES = 12;  // a warp's ring never grows beyond this
 constexpr int PIECE_SOFT = 24;  // groups a piece may grow to when that saves merge rounds
 constexpr float LAZY = 8.0f;   // the running maximum (log2 domain) may trail the true one by this much
 
@@ -180,91 +181,28 @@ __device__ __forceinline__ void merge_small(const float* pbase, int PS, int npie
   }
 }
 
-__global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
-  extern __shared__ __align__(128) unsigned char smem[];
+// The streaming of a warp's pieces.  DEEP: the CTA's ring stages are shared out among at most two
+// warps, the last stage of a warp's share holds the slot ids of its piece (one bulk copy of the
+// list segment), so that no copy waits for a global load of ids.  Otherwise: three stages per
+// warp, ids requested through registers two fires ahead.
+template <bool DEEP>
+__device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned char* smem, const int* off, const int* nin,
+                                              int U, int Ptot, int nWarps, int nall_rt, bool dyn, int pi, uint32_t bars_u32) {
   const State& st = p.st;
-  // Without `early` the kernel before this one may still be writing the lists this one reads.
-  if (!p.early) pdl_wait();
-  const int U = st.batch * st.H;
-  // ring stages, then one mbarrier per stage, then the split tables
-  const uint32_t bars_u32 = smem_u32(smem) + RING_BYTES;
-  int* off = reinterpret_cast<int*>(smem + RING_BYTES + NW * STAGES * 8);   // U + 1 piece prefix sums
-  int* nin = off + (U + 1);                                                  // U entry counts before the step
-  __shared__ int s_red[NW + 1];
-  __shared__ int s_mx[NW];
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
   const int G = p.G;
   const int PS = 16 + G * HD;
-
-  if (threadIdx.x < NW * STAGES) mbar_init(bars_u32 + threadIdx.x * 8, 1);
-  asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");   // made visible to the copy engine
-  // ---- every CTA derives the same split.  T = groups a piece may hold at most, chosen so that
-  // the pieces of all heads fit the grid's warps: sum ceil(g_u / T) <= Gtot / T + U <= nWarps.
-  const int nWarps = gridDim.x * NW;
-  int T;
-  {
-    int mine = 0, gmax = 0;
-    for (int u = tid; u < U; u += NT) {
-      const int uid = ((u / st.H) * st.L + p.layer) * st.H + (u % st.H);
-      const int n = p.n_in[uid];
-      nin[u] = n;
-      const int g = (n + p.append + GRP - 1) / GRP;
-      mine += g;
-      gmax = max(gmax, g);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
-    if (lane == 0) s_mx[w] = gmax;
-    int Gtot;
-    block_excl_scan(mine, s_red, Gtot);   // its barriers also publish s_mx
-    if (Gtot == 0) return;
-    for (int x = 0; x < NW; ++x) gmax = max(gmax, s_mx[x]);
-    T = (nWarps > U) ? (Gtot + (nWarps - U) - 1) / (nWarps - U) : 0x7fffffff;
-    // Small launches have warps to spare: pieces of up to PIECE_SOFT groups keep a unit at four
-    // pieces or fewer, which the merge handles in a single round of loads.
-    T = max(T, min(PIECE_SOFT, (gmax + 3) / 4));
-    T = max(T, GMIN);
-    int run = 0;
-    for (int b0 = 0; b0 < U; b0 += NT) {
-      const int u = b0 + tid;
-      int k = 0;
-      if (u < U) {
-        const int g = (nin[u] + p.append + GRP - 1) / GRP;
-        k = (T == 0x7fffffff) ? (g > 0) : (g + T - 1) / T;   // more heads than warps: one piece each
-      }
-      int tot;
-      const int ex = block_excl_scan(k, s_red, tot);
-      if (u < U) off[u] = run + ex;
-      run += tot;
-    }
-    if (tid == 0) off[U] = run;
-    __syncthreads();
-  }
-  const int Ptot = off[U];
-  // Which piece a warp takes.  When every warp gets at most one, pieces go to the warps in the
-  // order in which they become ready (one atomic each): CTAs that reach an SM late, because the
-  // kernel ahead held it longer, then find the pieces gone instead of finishing last.  The
-  // counter of the other parity is cleared for the next launch: all takes of the launch before
-  // this one happened before it let this one start.
-  const bool dyn = Ptot <= nWarps;
-  if (blockIdx.x == 0 && tid == 0) {
-    atomicExch(p.piece_ctr + (p.parity ^ 1), 0);
-    __threadfence();
-  }
-  int pi;
-  if (dyn) {
-    pi = 0;
-    if (lane == 0) pi = atomicAdd(p.piece_ctr + p.parity, 1);
-    pi = __shfl_sync(0xffffffffu, pi, 0);
-  } else {
-    pi = w * gridDim.x + blockIdx.x;   // ranks interleave over the CTAs
-  }
-  if (pi >= Ptot) return;
-
-  const uint32_t ring_u32 = smem_u32(smem) + w * (STAGES * STAGE_BYTES);
+  const int nall = DEEP ? nall_rt : STAGES;
+  constexpr bool ids_in_smem = DEEP;
+  const int nst = DEEP ? nall - 1 : STAGES;   // ring depth per working warp
+  (void)tid;
+  const uint32_t ring_u32 = smem_u32(smem) + w * (nall * STAGE_BYTES);   // w < apc whenever the warp has a piece
+  const uint32_t ids_u32 = ring_u32 + nst * STAGE_BYTES;
+  const uint32_t idbar = bars_u32 + (NW * STAGES + w) * 8;
+  uint32_t idphase = 0;
   const int gid = lane >> 2, tig = lane & 3;
   const int mi = lane >> 3, r8 = lane & 7;
-  const uint32_t bar0 = bars_u32 + w * (STAGES * 8);
+  const uint32_t bar0 = bars_u32 + w * (nall * 8);
   // ldmatrix row addresses inside a stage: K tile of k-step ks at kb + 32 ks, V tile of channel
   // tile mt at vb + 32 mt
   const uint32_t kb = (uint32_t)(((mi & 1) * 8 + r8) * ENTRY_STRIDE + (mi >> 1) * 16);
@@ -297,10 +235,11 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
     const int* list = st.list_slot + mb;
     const unsigned char* pool = st.pool + (size_t)seq * st.slots_per_seq * SLOT_BYTES;
 
-    // ---- issuing side
+    // ---- issuing side.  The lane that holds an entry's slot id issues its copy.  The ids come
+    // from shared memory (deep rings) or are requested two fires before they are needed.
     auto slots_of = [&](int idx) {   // lane e: pool slot of entry 16 idx + e (0 past the end)
       const int i = idx * GRP + lane;
-      return (lane < GRP && i < n_tot) ? list[i] : 0;
+      return (lane < GRP && idx < hi && i < n_tot) ? list[i] : 0;
     };
     auto fire = [&](int idx, int slot, uint32_t stage, uint32_t bar) {
       const int valid = min(GRP, n_tot - idx * GRP);
@@ -322,22 +261,40 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
       }
     };
-    // groups flow through the ring, STAGES-1 of them in flight; the slot ids of a group are
-    // requested two fires before they are needed
+    // groups flow through the ring, nst-1 of them in flight
     int next = lo;
-    int sl0 = slots_of(lo), sl1 = (lo + 1 < hi) ? slots_of(lo + 1) : 0;
+    int sl0 = 0, sl1 = 0;
+    const bool ids_here = ids_in_smem && (hi - lo) * GRP * 4 <= STAGE_BYTES;   // else: ids through registers
+    if (ids_here) {
+      // the list positions of groups lo .. hi-1 are contiguous and 64-byte aligned
+      if (lane == 0) {
+        mbar_expect_tx(idbar, (uint32_t)(hi - lo) * GRP * 4);
+        bulk_g2s(ids_u32, list + (size_t)lo * GRP, (uint32_t)(hi - lo) * GRP * 4, idbar);
+      }
+      if (!mbar_wait_bounded(idbar, idphase)) {
+        if (lane == 0) atomicOr(st.errword, ERR_COPY_TIMEOUT);
+        return;
+      }
+      idphase ^= 1u;
+    } else {
+      sl0 = slots_of(lo); sl1 = slots_of(lo + 1);
+    }
     auto fire_next = [&]() {
       if (next < hi) {
-        const int sl = sl0;
-        sl0 = sl1;
-        if (next + 2 < hi) sl1 = slots_of(next + 2);
-        fire(next, sl, ring_u32 + fsi * STAGE_BYTES, bar0 + fsi * 8);
+        int slot = sl0;
+        if (ids_here) {
+          asm volatile("ld.shared.b32 %0, [%1];\n" : "=r"(slot) : "r"(ids_u32 + (uint32_t)((next - lo) * GRP + (lane & 15)) * 4));
+        } else {
+          sl0 = sl1;
+          sl1 = slots_of(next + 2);
+        }
+        fire(next, slot, ring_u32 + fsi * STAGE_BYTES, bar0 + fsi * 8);
         ++next;
-        fsi = (fsi + 1 == STAGES) ? 0 : fsi + 1;
+        fsi = (fsi + 1 == nst) ? 0 : fsi + 1;
       }
     };
 #pragma unroll 1
-    for (int s = 0; s < STAGES - 1; ++s) fire_next();
+    for (int s = 0; s < nst - 1; ++s) fire_next();
     // everything above reads only the cache and its lists; the call's inputs (q here, the
     // arriving row inside fire) may come from the kernel ahead in the stream
     if (!waited) { pdl_wait(); waited = true; }
@@ -366,7 +323,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
         // a copy did not land: flag it, give the other stages' copies their chance to land in
         // this CTA's memory while it still belongs to us, and leave the head unfinished
         if (lane == 0) atomicOr(st.errword, ERR_COPY_TIMEOUT);
-        for (int s = 0; s < STAGES; ++s)
+        for (int s = 0; s < nst; ++s)
           if (s != csi) mbar_wait_bounded(bar0 + s * 8, (phases >> s) & 1u);
         return;
       }
@@ -449,10 +406,42 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
           mma_bf16(o[mt], a, rr0, rr1);
         }
       }
-      csi = (csi + 1 == STAGES) ? 0 : csi + 1;
+      csi = (csi + 1 == nst) ? 0 : csi + 1;
       __syncwarp();   // the stage is free for the fire of the next iteration
     }
 
+    if (npieces == 1) {
+      // ---- the whole head was this warp's: normalise and write `out` from the accumulators
+      float ls0 = l0, ls1 = l1;
+#pragma unroll
+      for (int x = 4; x < 32; x <<= 1) {
+        ls0 += __shfl_xor_sync(0xffffffffu, ls0, x);
+        ls1 += __shfl_xor_sync(0xffffffffu, ls1, x);
+      }
+      const float i0 = 1.0f / ls0, i1 = 1.0f / ls1;
+      const int h0 = 2 * tig, h1 = 2 * tig + 1;
+      __nv_bfloat16* ob = p.out + (size_t)u * G * HD + gid;
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        if (h0 < G) {
+          ob[h0 * HD + 16 * mt] = __float2bfloat16_rn(o[mt][0] * i0);
+          ob[h0 * HD + 16 * mt + 8] = __float2bfloat16_rn(o[mt][2] * i0);
+        }
+        if (h1 < G) {
+          ob[h1 * HD + 16 * mt] = __float2bfloat16_rn(o[mt][1] * i1);
+          ob[h1 * HD + 16 * mt + 8] = __float2bfloat16_rn(o[mt][3] * i1);
+        }
+      }
+      if (gid == 0 && p.track) {   // reference point and normaliser of the step's softmax, for the LRFU kernel
+        if (h0 < G) { p.sc.mfin[u * (2 * QH) + h0] = m0; p.sc.mfin[u * (2 * QH) + QH + h0] = ls0; }
+        if (h1 < G) { p.sc.mfin[u * (2 * QH) + h1] = m1; p.sc.mfin[u * (2 * QH) + QH + h1] = ls1; }
+      }
+      if (lane == 0) {
+        atomicAdd(&st.counters[0], (unsigned long long)n_tot);
+        if (!p.track) keep_and_refill(st, p.n_out, uid, seq, n_tot, p.append != 0);
+      }
+      continue;
+    }
     // ---- publish the piece's partial and take a ticket
     float* part = p.sc.partials + ((size_t)u * p.sc.pmax + piece) * PS;
     {
@@ -559,6 +548,102 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
       if (!p.track) keep_and_refill(st, p.n_out, uid, seq, n_tot, p.append != 0);
     }
   }
+}
+
+__global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const State& st = p.st;
+  // Without `early` the kernel before this one may still be writing the lists this one reads.
+  if (!p.early) pdl_wait();
+  const int U = st.batch * st.H;
+  // ring stages, then one mbarrier per stage, then the split tables
+  const uint32_t bars_u32 = smem_u32(smem) + RING_BYTES;
+  int* off = reinterpret_cast<int*>(smem + RING_BYTES + (NW * STAGES + NW) * 8);   // U + 1 piece prefix sums
+  int* nin = off + (U + 1);                                                  // U entry counts before the step
+  __shared__ int s_red[NW + 1];
+  __shared__ int s_mx[NW];
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  const int G = p.G;
+  const int PS = 16 + G * HD;
+
+  if (threadIdx.x < NW * STAGES + NW) mbar_init(bars_u32 + threadIdx.x * 8, 1);
+  asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");   // made visible to the copy engine
+  // ---- every CTA derives the same split.  T = groups a piece may hold at most, chosen so that
+  // the pieces of all heads fit the grid's warps: sum ceil(g_u / T) <= Gtot / T + U <= nWarps.
+  const int nWarps = gridDim.x * NW;
+  int T;
+  {
+    int mine = 0, gmax = 0;
+    for (int u = tid; u < U; u += NT) {
+      const int uid = ((u / st.H) * st.L + p.layer) * st.H + (u % st.H);
+      const int n = p.n_in[uid];
+      nin[u] = n;
+      const int g = (n + p.append + GRP - 1) / GRP;
+      mine += g;
+      gmax = max(gmax, g);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
+    if (lane == 0) s_mx[w] = gmax;
+    int Gtot;
+    block_excl_scan(mine, s_red, Gtot);   // its barriers also publish s_mx
+    if (Gtot == 0) return;
+    for (int x = 0; x < NW; ++x) gmax = max(gmax, s_mx[x]);
+    T = (nWarps > U) ? (Gtot + (nWarps - U) - 1) / (nWarps - U) : 0x7fffffff;
+    // (Pieces are not made longer than that on purpose: issuing the 16 bulk copies of a group
+    // blocks the issuing warp for about half a microsecond, as long as the group's MMAs take, so
+    // the copy rate of a launch grows with the number of warps that stream.)
+    // Small launches: pieces of up to PIECE_SOFT groups keep a unit at four pieces or fewer,
+    // which the merge handles in a single round of loads.
+    T = max(T, min(PIECE_SOFT, (gmax + 3) / 4));
+    T = max(T, GMIN);
+    int run = 0;
+    for (int b0 = 0; b0 < U; b0 += NT) {
+      const int u = b0 + tid;
+      int k = 0;
+      if (u < U) {
+        const int g = (nin[u] + p.append + GRP - 1) / GRP;
+        k = (T == 0x7fffffff) ? (g > 0) : (g + T - 1) / T;   // more heads than warps: one piece each
+      }
+      int tot;
+      const int ex = block_excl_scan(k, s_red, tot);
+      if (u < U) off[u] = run + ex;
+      run += tot;
+    }
+    if (tid == 0) off[U] = run;
+    __syncthreads();
+  }
+  const int Ptot = off[U];
+  // Which piece a warp takes.  When every warp gets at most one, pieces go to the warps in the
+  // order in which they become ready (one atomic each): CTAs that reach an SM late, because the
+  // kernel ahead held it longer, then find the pieces gone instead of finishing last.  The
+  // counter of the other parity is cleared for the next launch: all takes of the launch before
+  // this one happened before it let this one start.
+  // apc = pieces a CTA gets at most; its warps with a piece share the CTA's ring stages
+  const int apc = min(NW, (Ptot + (int)gridDim.x - 1) / (int)gridDim.x);
+  // A warp with four stages or more gives the last one to the slot ids of its piece (one bulk
+  // copy of the list segment), so that no copy waits for a global load of ids.
+  // Deep rings pay when at most two warps of a CTA stream (their few warps are then bound by
+  // latency); with more, three stages and all eight warps competing for the pieces are faster.
+  const int nall = apc <= 2 ? min(MAX_STAGES + 1, (NW * STAGES) / apc) : STAGES;
+  const bool dyn = Ptot <= nWarps;
+  if (dyn && nall > STAGES && w >= apc) return;   // a deep ring: the CTA's stages are shared out among its first apc warps
+  if (blockIdx.x == 0 && tid == 0) {
+    atomicExch(p.piece_ctr + (p.parity ^ 1), 0);
+    __threadfence();
+  }
+  int pi;
+  if (dyn) {
+    pi = 0;
+    if (lane == 0) pi = atomicAdd(p.piece_ctr + p.parity, 1);
+    pi = __shfl_sync(0xffffffffu, pi, 0);
+  } else {
+    pi = w * gridDim.x + blockIdx.x;   // ranks interleave over the CTAs
+  }
+  if (pi >= Ptot) return;
+
+  if (nall > STAGES) stream_pieces<true>(p, smem, off, nin, U, Ptot, nWarps, nall, dyn, pi, bars_u32);
+  else stream_pieces<false>(p, smem, off, nin, U, Ptot, nWarps, nall, dyn, pi, bars_u32);
 }
 
 }  // namespace ckv

@@ -322,6 +322,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   // list positions per head: entries up to the largest budget plus the arriving one and the
   // answer-stage tail, plus the spare; FullKV keeps every token
   h->cap = evict ? c.max_budget + 1 + c.max_answer_tokens + 1 : c.max_context + 1;
+  h->cap = (h->cap + GRP - 1) / GRP * GRP;   // whole 16-entry groups: a piece's slot ids are one aligned bulk copy
   h->slots_per_seq = (long long)c.n_layers * c.n_kv_heads *
                      (evict ? (long long)c.budget_per_head + 1 + c.max_answer_tokens : (long long)c.max_context + 1);
   if (h->slots_per_seq > 0x7fffffffLL) { g_create_err = "more than 2^31 slots per sequence"; delete h; return CRYSTALKV_EINVAL; }
@@ -351,7 +352,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   cudaDeviceProp prop;
   CKC(cudaGetDeviceProperties(&prop, c.device));
   h->num_sms = prop.multiProcessorCount;
-  h->smem = RING_BYTES + NW * STAGES * 8 + (size_t)(2 * h->U + 1) * sizeof(int);
+  h->smem = RING_BYTES + (NW * STAGES + NW) * 8 + (size_t)(2 * h->U + 1) * sizeof(int);
   int bps = 0;
   CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem));
   CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
