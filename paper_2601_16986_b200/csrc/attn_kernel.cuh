@@ -508,6 +508,14 @@ __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned ch
           for (int h = 0; h < 4; ++h) put(g0 + h, mm[h], L[h], acc[h]);
         }
       }
+    } else if (npieces <= 8) {   // two heads x eight pieces per round
+      for (int g0 = 0; g0 < G; g0 += 2) {
+        float mm[2], L[2];
+        float4 acc[2];
+        merge_small<2, 8>(pbase, PS, npieces, g0, G, lane, mm, L, acc);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) put(g0 + h, mm[h], L[h], acc[h]);
+      }
     } else {
       const int hh = lane & 7, pl = lane >> 3;   // header phase: lane = (piece mod 4, head)
       float mm = -INFINITY, Ls = 0.f;

@@ -142,11 +142,30 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       }
     }
   } else if (EPT > 0) {
+    // batches of four entries: their rows are requested together (clamped index, no branch)
 #pragma unroll
-    for (int k = 0; k < R; ++k) {
-      const int i = tid + k * NT;
-      pmr[k] = 0.f;
-      if (k < kmax && i < n) pmr[k] = pbar_of(i);
+    for (int k = 0; k < R; ++k) pmr[k] = 0.f;
+#pragma unroll
+    for (int k0 = 0; k0 < R; k0 += 4) {
+      if (k0 < kmax) {
+        float4 ra[4], rb[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int i = min(tid + (k0 + j) * NT, n - 1);
+          ra[j] = ld_f32x4(S + (size_t)i * QH);
+          rb[j] = (G > 4) ? ld_f32x4(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (k0 + j < R) {
+            const float sv[8] = {ra[j].x, ra[j].y, ra[j].z, ra[j].w, rb[j].x, rb[j].y, rb[j].z, rb[j].w};
+            float pm = 0.f;
+#pragma unroll
+            for (int g = 0; g < G; ++g) pm = fmaf(expf(sv[g] - mx[g]), invl[g], pm);
+            pmr[k0 + j] = (tid + (k0 + j) * NT < n) ? pm : 0.f;
+          }
+        }
+      }
     }
   } else {
     for (int i = tid; i < n; i += NT) pbar[i] = pbar_of(i);
@@ -386,13 +405,26 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       if (less) { bk0 = c0; bk1 = c1; bk2 = c2; bidx = i; }
     }
   };
-  if (EPT > 8) {   // many entries per thread: one at a time keeps the registers down
+  if (EPT > 8) {   // many entries per thread: four at a time, their stored state requested together
 #pragma unroll
-    for (int k = 0; k < R; ++k) {
-      const int i = tid + k * NT;
-      if (k < kmax && i < n) {
-        const int tau = st.meta_tau[mb + i];
-        update(i, pmr[k], st.meta_pos[mb + i], tau, st.meta_crf[mb + i], __ldg(st.tab + (p.t - tau)));
+    for (int k0 = 0; k0 < R; k0 += 4) {
+      if (k0 < kmax) {
+        int pos4[4], tau4[4];
+        float crf4[4], dec4[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const size_t i = mb + min(tid + (k0 + j) * NT, n - 1);
+          pos4[j] = ld_i32(st.meta_pos + i);
+          tau4[j] = ld_i32(st.meta_tau + i);
+          crf4[j] = ld_f32(st.meta_crf + i);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dec4[j] = __ldg(st.tab + (p.t - min(tau4[j], p.t)));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int i = tid + (k0 + j) * NT;
+          if (k0 + j < R && i < n) update(i, pmr[k0 + j < R ? k0 + j : 0], pos4[j], tau4[j], crf4[j], dec4[j]);
+        }
       }
     }
   } else if (EPT > 0) {
