@@ -18,7 +18,9 @@
  * and a library scaled-dot-product attention; the hit mask against subset
  * enumeration; CRF against the closed form of Section 5.2 and the lambda = 0 / 1
  * limits; eviction against a full sort; Algorithm 2 against hand examples and its
- * invariants; "budget = entries per head" against Table 1's HBM-saving column.
+ * invariants; "budget = entries per head" against Table 1's HBM-saving column; the
+ * observation-window prefill, the buffered eviction cadence and the literal early
+ * return against the same definition-level simulator as the plain trajectory.
  * Whole trajectories (which tokens survive thousands of steps) have no value printed
  * in the paper: parity unpinned for those beyond the per-step pins above.
  *
@@ -45,6 +47,8 @@ typedef struct {
     int32_t mode;
     float top_p, lambda, sm_scale;
     double tie_eps; /* relative window for the tie log (1e-6) */
+    int32_t evict_every;    /* m: step 4 runs once a head is m entries over its budget (0, 1: every step) */
+    int32_t literal_return; /* 1: Algorithm 1's first line taken literally (nothing runs while Len(K) < B) */
 } okv_config;
 
 typedef struct {
@@ -296,13 +300,19 @@ static int evict_lowest(okv_unit *u, const float *crf_temp, int k, double rel_ep
  * Reading (GQA): the cache, CRF and budget belong to the KV head; the hit mask is
  * taken from the mean of the group's G probability vectors, itself a distribution.
  * Reading (step 1 early return): scoring and CRF tracking run on every think step;
- * only the eviction is gated by Len(K) > B.
+ * only the eviction is gated by Len(K) > B.  With literal_return the algorithm's first
+ * line is taken as printed instead: while Len(K) < B steps 1-4 are all skipped.
+ * Reading (buffered cadence, evict_every = m > 1): step 4 waits until the head is m
+ * entries over its budget and then removes all of them at once (k = m per call).
+ * hold: steps 1-3 only (the observation-window replay of the prompt evicts once, at
+ * its last query).
  * y (may be NULL): [G][d] fp32 attention output.
  */
 static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, int t,
-                      int track, float *y) {
+                      int track, int hold, float *y) {
     okv_unit *u = unit_of(o, seq, layer, head);
     int n = u->n, d = o->c.head_dim, G = o->c.n_q_heads / o->c.n_kv_heads;
+    if (track && o->c.literal_return && n < u->budget) track = 0;
     const double **kr = (const double **)malloc((size_t)n * sizeof(void *));
     const double **vr = (const double **)malloc((size_t)n * sizeof(void *));
     for (int i = 0; i < n; ++i) { kr[i] = u->e[i].k; vr[i] = u->e[i].v; }
@@ -328,7 +338,9 @@ static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, i
         okv_hit_mask(pbar, pos, n, (double)o->c.top_p, hit, o->c.tie_eps, &near);
         if (near) log_tie(o, layer, seq, head, t, OKV_TIE_NUCLEUS);
         crf_update(o, u, t, hit, ct);
-        if (evict_lowest(u, ct, n - u->budget, o->c.tie_eps))
+        int m = o->c.evict_every > 1 ? o->c.evict_every : 1;
+        int over = n - u->budget;
+        if (!hold && over >= m && evict_lowest(u, ct, over, o->c.tie_eps))
             log_tie(o, layer, seq, head, t, OKV_TIE_EVICT);
         free(pbar); free(pos); free(hit); free(ct);
     }
@@ -388,7 +400,39 @@ int okv_prefill(okv *o, int layer, const uint16_t *k, const uint16_t *v, const u
                 unit_append(o, u, i, k + off, v + off, 0.0f, P - 1);
             }
             const uint16_t *q = q_last + ((size_t)b * c->n_q_heads + (size_t)h * G) * d;
-            if (track) lrfu_pass(o, b, layer, h, q, P - 1, 1, NULL);
+            if (track) lrfu_pass(o, b, layer, h, q, P - 1, 1, 0, NULL);
+        }
+    o->t_layer[layer] = P - 1;
+    return OKV_OK;
+}
+
+/*
+ * Prompt with an observation window: k, v [batch][P][H][d]; q_win [W][batch][Hq][d] are
+ * the queries of prompt tokens P-W .. P-1; y_win (may be NULL) [W][batch][Hq][d] their
+ * causal attention outputs.  Reading: the last W prompt tokens are replayed as decode
+ * steps whose eviction is deferred: token i arrives with CRF 0 and tau = i, the query
+ * of token t in the window attends to tokens 0..t and runs Algorithm 1 steps 1-3 at
+ * time t, and step 4 runs once, after the last query (t = P-1).
+ */
+int okv_prefill_window(okv *o, int layer, const uint16_t *k, const uint16_t *v, const uint16_t *q_win,
+                       int P, int W, float *y_win) {
+    const okv_config *c = &o->c;
+    if (layer < 0 || layer >= c->n_layers || P < 1 || W < 1 || W > P || o->t_layer[layer] >= 0) return OKV_ERR;
+    int H = c->n_kv_heads, d = c->head_dim, G = c->n_q_heads / H;
+    int track = (c->mode == OKV_MODE_EVICT);
+    size_t qn = (size_t)c->batch * c->n_q_heads * d;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < c->batch; ++b)
+        for (int h = 0; h < H; ++h) {
+            okv_unit *u = unit_of(o, b, layer, h);
+            for (int i = 0; i < P; ++i) {
+                size_t off = (((size_t)b * P + i) * H + h) * d;
+                unit_append(o, u, i, k + off, v + off, 0.0f, i);
+                int w = i - (P - W);
+                if (w < 0) continue;
+                size_t qo = (size_t)w * qn + ((size_t)b * c->n_q_heads + (size_t)h * G) * d;
+                lrfu_pass(o, b, layer, h, q_win + qo, i, track, i < P - 1, y_win ? y_win + qo : NULL);
+            }
         }
     o->t_layer[layer] = P - 1;
     return OKV_OK;
@@ -415,7 +459,7 @@ int okv_decode_step(okv *o, int layer, const uint16_t *q, const uint16_t *k_new,
             size_t kvo = ((size_t)b * H + h) * d;
             unit_append(o, u, t, k_new + kvo, v_new + kvo, 0.0f, t);
             size_t qo = ((size_t)b * c->n_q_heads + (size_t)h * G) * d;
-            lrfu_pass(o, b, layer, h, q + qo, t, track, out + qo);
+            lrfu_pass(o, b, layer, h, q + qo, t, track, 0, out + qo);
         }
     o->t_layer[layer] = t;
     return OKV_OK;

@@ -23,7 +23,8 @@ class _Cfg(C.Structure):
                 ("head_dim", C.c_int32), ("batch", C.c_int32), ("budget_per_head", C.c_int32),
                 ("min_budget", C.c_int32), ("max_budget", C.c_int32), ("max_context", C.c_int32),
                 ("mode", C.c_int32), ("top_p", C.c_float), ("lam", C.c_float),
-                ("sm_scale", C.c_float), ("tie_eps", C.c_double)]
+                ("sm_scale", C.c_float), ("tie_eps", C.c_double),
+                ("evict_every", C.c_int32), ("literal_return", C.c_int32)]
 
 
 @dataclass
@@ -42,6 +43,8 @@ class OracleConfig:
     lam: float = 0.6
     sm_scale: float = 0.0        # 0 -> 1/sqrt(head_dim)
     tie_eps: float = 1e-6
+    evict_every: int = 1         # m: evict once a head is m entries over its budget
+    literal_return: int = 0      # 1: no tracking while a head is below its budget (Algorithm 1, first line)
 
 
 _lib = None
@@ -57,6 +60,7 @@ def _load():
         lib.okv_destroy.argtypes = [vp]
         lib.okv_set_stage.argtypes = [vp, i32]
         lib.okv_prefill.argtypes = [vp, i32, vp, vp, vp, i32]
+        lib.okv_prefill_window.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
         lib.okv_decode_step.argtypes = [vp, i32, vp, vp, vp, vp]
         lib.okv_rebudget.argtypes = [vp]
         lib.okv_get_retained.argtypes = [vp, i32, i32, i32, vp, i32]
@@ -132,7 +136,7 @@ class Oracle:
         max_b = cfg.max_budget or cfg.budget_per_head * cfg.n_layers * cfg.n_kv_heads
         self._c = _Cfg(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.batch,
                        cfg.budget_per_head, cfg.min_budget, max_b, cfg.max_context, cfg.mode,
-                       cfg.top_p, cfg.lam, cfg.sm_scale, cfg.tie_eps)
+                       cfg.top_p, cfg.lam, cfg.sm_scale, cfg.tie_eps, cfg.evict_every, cfg.literal_return)
         self._h = lib.okv_create(C.byref(self._c))
         if not self._h:
             raise ValueError("oracle: bad config")
@@ -159,6 +163,17 @@ class Oracle:
         rc = self._lib.okv_prefill(self._h, layer, _p(kb), _p(vb), _p(qb), P)
         if rc:
             raise RuntimeError("oracle prefill failed")
+
+    def prefill_window(self, layer, k, v, q_win) -> np.ndarray:
+        """k, v [batch,P,H,d]; q_win [W,batch,Hq,d] (bf16), the queries of the last W prompt
+        tokens -> their causal attention outputs [W,batch,Hq,d] float32."""
+        P, W = k.shape[1], q_win.shape[0]
+        kb, vb, qb = _bits(k), _bits(v), _bits(q_win)
+        y = np.zeros(q_win.shape, dtype=np.float32)
+        rc = self._lib.okv_prefill_window(self._h, layer, _p(kb), _p(vb), _p(qb), P, W, _p(y))
+        if rc:
+            raise RuntimeError("oracle prefill_window failed")
+        return y
 
     def decode_step(self, layer, q, k_new, v_new) -> np.ndarray:
         """-> out [batch,Hq,d] float32."""

@@ -53,8 +53,10 @@ def brute_hits(pbar, p):
 class BruteUnit:
     """One (sequence, layer, kv-head) cache simulated from definitions."""
 
-    def __init__(self, budget, lam, top_p, scale):
+    def __init__(self, budget, lam, top_p, scale, evict_every=1, literal_return=False):
         self.B, self.lam, self.p, self.scale = budget, lam, top_p, scale
+        self.m = max(1, evict_every)   # eviction waits until the head is m entries over its budget
+        self.literal = literal_return  # nothing of Algorithm 1 runs while the head is below its budget
         self.pos, self.K, self.V = [], [], []
         self.hits = []     # per entry: list of hit times
         self.arrival = []  # per entry: arrival time (tau before the first hit)
@@ -70,13 +72,13 @@ class BruteUnit:
     def last(self, i):
         return self.hits[i][-1] if self.hits[i] else self.arrival[i]
 
-    def step(self, q, t, track=True):
+    def step(self, q, t, track=True, evict=True):
         """Attention at time t; returns (y, min_gap) where min_gap is the smallest
         relative distance of any decision from flipping (for skipping near-ties)."""
         K, V = np.stack(self.K), np.stack(self.V)
         prob, y = naive_attention(q, K, V, self.scale)
         gap = np.inf
-        if track:
+        if track and not (self.literal and len(self.pos) < self.B):
             pbar = prob.mean(axis=0)
             (S, nwin) = brute_hits(list(pbar), self.p)
             srt = np.sort(pbar)[::-1]
@@ -88,7 +90,7 @@ class BruteUnit:
             for i in S:
                 self.hits[i].append(t)
             n = len(self.pos)
-            if n > self.B:
+            if evict and n - self.B >= self.m:
                 keys = [(self.crf(i, t), self.last(i), self.pos[i], i) for i in range(n)]
                 keys.sort()
                 kk = n - self.B

@@ -339,3 +339,104 @@ def test_answer_stage_freezes_the_think_cache():
     assert len(after) == len(before) + 5
     assert (after[:len(before)] == before).all()          # nothing updated, nothing evicted
     o.close()
+
+
+# ------------------------------------------------------------ variants of Algorithm 1's schedule
+def _compare_unit(o, u, h, tol=1e-5):
+    assert o.get_retained(0, 0, h).tolist() == sorted(u.pos)
+    st = o.export_state(0, 0, h)
+    crf = st[:, 1].view(np.float32)
+    for r, i in enumerate(np.argsort(u.pos)):
+        tau = u.last(i)
+        assert st[r, 2] == tau
+        np.testing.assert_allclose(crf[r], u.crf(i, tau), rtol=tol, atol=0)
+
+
+@pytest.mark.parametrize("W,P,B", [(1, 10, 6), (4, 12, 7), (6, 6, 4), (5, 9, 20)])
+def test_window_prefill_matches_brute_force(W, P, B):
+    """Algorithm 1 over an observation window of the prompt: the last W prompt tokens replayed
+    as causal steps with steps 1-3 only, one eviction after the last query; then decode."""
+    G = 2
+    w = tiny(n_q_heads=2 * G, n_kv_heads=2, prompt=P, think_steps=12, budget_per_head=B, seed=41 + W)
+    o = make_oracle(w)
+    scale = 1.0 / np.sqrt(w.head_dim)
+    k, v = w.prompt_kv(0)
+    qw = w.queries(0, list(range(P - W, P))).transpose(0, 1).contiguous()   # [W, batch, Hq, d]
+    y = o.prefill_window(0, k, v, qw)
+    units = []
+    for h in range(2):
+        u = BruteUnit(B, float(np.float32(w.lam)), float(np.float32(w.top_p)), scale)
+        for i in range(P):
+            u.append(i, f64(k[0, i, h]), f64(v[0, i, h]), i)
+            if i >= P - W:
+                yy, gap = u.step(f64(qw[i - (P - W), 0, h * G:(h + 1) * G]), i, evict=(i == P - 1))
+                if gap < 1e-4:
+                    pytest.skip("near-tie in the brute-force reference; pick another seed")
+                np.testing.assert_allclose(y[i - (P - W), 0, h * G:(h + 1) * G], yy, rtol=1e-5, atol=1e-6)
+        assert len(u.pos) == min(P, B)
+        _compare_unit(o, u, h)
+        units.append(u)
+    for t in range(P, P + w.think_steps):
+        q, kn, vn = w.step_inputs(0, t)
+        o.decode_step(0, q, kn, vn)
+        for h, u in enumerate(units):
+            u.append(t, f64(kn[0, h]), f64(vn[0, h]), t)
+            _, gap = u.step(f64(q[0, h * G:(h + 1) * G]), t)
+            if gap < 1e-4:
+                pytest.skip("near-tie in the brute-force reference; pick another seed")
+            _compare_unit(o, u, h)
+    o.close()
+
+
+def test_window_of_one_keeps_what_the_last_query_prefill_keeps():
+    """W = 1 differs from the Q^last prefill only in the tau recorded for entries never hit."""
+    w = tiny(prompt=14, budget_per_head=6, seed=3)
+    k, v = w.prompt_kv(0)
+    ql = w.queries(0, [w.prompt - 1])[:, 0]
+    a, b = make_oracle(w), make_oracle(w)
+    a.prefill(0, k, v, ql)
+    b.prefill_window(0, k, v, ql.unsqueeze(0))
+    for h in range(2):
+        assert a.get_retained(0, 0, h).tolist() == b.get_retained(0, 0, h).tolist()
+        sa, sb = a.export_state(0, 0, h), b.export_state(0, 0, h)
+        assert (sa[:, 1] == sb[:, 1]).all()
+        hit = sa[:, 1].view(np.float32) > 0
+        assert (sa[hit, 2] == sb[hit, 2]).all() and (sb[~hit, 2] == sb[~hit, 0]).all()
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("m,literal", [(4, 0), (3, 1), (1, 1), (7, 0)])
+def test_buffered_cadence_and_literal_return_match_brute_force(m, literal):
+    """Eviction every m entries (k = m per call) and Algorithm 1's first line as printed
+    (no scoring while Len(K) < B) against the simulator built from the definitions."""
+    G = 2
+    w = tiny(n_q_heads=2 * G, n_kv_heads=2, prompt=5, think_steps=36, budget_per_head=9, seed=50 + m)
+    o = make_oracle(w, evict_every=m, literal_return=literal)
+    scale = 1.0 / np.sqrt(w.head_dim)
+    k, v = w.prompt_kv(0)
+    qlast = w.queries(0, [w.prompt - 1])[:, 0]
+    o.prefill(0, k, v, qlast)
+    units, sizes = [], set()
+    for h in range(2):
+        u = BruteUnit(w.budget_per_head, float(np.float32(w.lam)), float(np.float32(w.top_p)), scale,
+                      evict_every=m, literal_return=bool(literal))
+        for i in range(w.prompt):
+            u.append(i, f64(k[0, i, h]), f64(v[0, i, h]), w.prompt - 1)
+        u.step(f64(qlast[0, h * G:(h + 1) * G]), w.prompt - 1)
+        if literal:
+            assert not any(u.hits)      # the prompt is shorter than the budget: nothing was scored
+        units.append(u)
+    for t in range(w.prompt, w.prompt + w.think_steps):
+        q, kn, vn = w.step_inputs(0, t)
+        out = o.decode_step(0, q, kn, vn)
+        for h, u in enumerate(units):
+            u.append(t, f64(kn[0, h]), f64(vn[0, h]), t)
+            y, gap = u.step(f64(q[0, h * G:(h + 1) * G]), t)
+            if gap < 1e-4:
+                pytest.skip("near-tie in the brute-force reference; pick another seed")
+            np.testing.assert_allclose(out[0, h * G:(h + 1) * G], y, rtol=1e-5, atol=1e-6)
+            _compare_unit(o, u, h)
+            sizes.add(len(u.pos))
+    assert max(sizes) == w.budget_per_head + m - 1      # the buffer fills before it is emptied
+    assert w.budget_per_head in sizes
+    o.close()
