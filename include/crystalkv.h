@@ -65,6 +65,10 @@ typedef struct {
   float sm_scale;          /* logit scale; 0 = 1/sqrt(head_dim) */
   int32_t mode;            /* CRYSTALKV_MODE_* */
   int32_t device;          /* CUDA device ordinal */
+  int32_t evict_every;     /* m: Algorithm 1 step 4 waits until a head is m entries over its budget and then
+                              removes all of them in one call (k = m); 0 or 1 = every step.  At most 4096. */
+  int32_t literal_return;  /* 1: Algorithm 1's first line as printed: while Len(K) < B of a head nothing
+                              of the algorithm runs for it (no hit mask, no CRF update); 0 = track always */
 } crystalkv_config_t;
 
 /*
@@ -87,6 +91,23 @@ int crystalkv_destroy(crystalkv_t* h);
  */
 int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v,
                       const void* q_last, int P, void* stream);
+
+/*
+ * Loads a prompt into one layer and replays Algorithm 1 over an observation window: the
+ * queries of the last W prompt tokens, in order.  Token i arrives with CRF 0 and tau = i;
+ * the query of token t (P-W <= t <= P-1) attends to tokens 0..t (causal) and runs steps 1-3
+ * at time t; step 4 runs once, after the last query, and brings every head down to its budget.
+ * W = 1 retains what crystalkv_prefill retains (tau of never-hit entries is their position
+ * instead of P-1).
+ *   k, v       dev [batch][P][H][128]
+ *   q_window   dev [W][batch][Hq][128]   queries of tokens P-W .. P-1
+ *   out_window dev [W][batch][Hq][128]   their attention outputs, or NULL
+ * All buffers belong to the caller and must stay valid until the work queued on `stream`
+ * has run.  1 <= W <= P; P as for crystalkv_prefill.  FullKV mode: only the insertion
+ * (and out_window, if asked for, stays untouched).  Errors: EINVAL; ESTATE if the layer was prefilled.
+ */
+int crystalkv_prefill_window(crystalkv_t* h, int layer, const void* k, const void* v,
+                             const void* q_window, int P, int W, void* out_window, void* stream);
 
 /*
  * One decode step of one layer for all sequences (Section 2.2 attention fused with

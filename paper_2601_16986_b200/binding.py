@@ -33,7 +33,8 @@ class _Cfg(C.Structure):
                 ("head_dim", C.c_int32), ("batch", C.c_int32), ("dtype", C.c_int32),
                 ("budget_per_head", C.c_int32), ("min_budget", C.c_int32), ("max_budget", C.c_int32),
                 ("max_answer_tokens", C.c_int32), ("max_context", C.c_int32), ("top_p", C.c_float),
-                ("lam", C.c_float), ("sm_scale", C.c_float), ("mode", C.c_int32), ("device", C.c_int32)]
+                ("lam", C.c_float), ("sm_scale", C.c_float), ("mode", C.c_int32), ("device", C.c_int32),
+                ("evict_every", C.c_int32), ("literal_return", C.c_int32)]
 
 
 @dataclass
@@ -54,6 +55,8 @@ class Config:
     mode: int = EVICT
     device: int = 0
     dtype: int = BF16
+    evict_every: int = 1
+    literal_return: int = 0
 
 
 def declared_symbols():
@@ -78,6 +81,7 @@ def load_library():
     lib.crystalkv_create.argtypes = [C.POINTER(_Cfg), C.POINTER(vp)]
     lib.crystalkv_destroy.argtypes = [vp]
     lib.crystalkv_prefill.argtypes = [vp, i32, vp, vp, vp, i32, vp]
+    lib.crystalkv_prefill_window.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, vp]
     lib.crystalkv_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.crystalkv_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.crystalkv_set_stage.argtypes = [vp, i32]
@@ -123,7 +127,8 @@ class CrystalKV:
         self.cfg = cfg
         c = _Cfg(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.batch, cfg.dtype,
                  cfg.budget_per_head, cfg.min_budget, cfg.max_budget, cfg.max_answer_tokens,
-                 cfg.max_context, cfg.top_p, cfg.lam, cfg.sm_scale, cfg.mode, cfg.device)
+                 cfg.max_context, cfg.top_p, cfg.lam, cfg.sm_scale, cfg.mode, cfg.device,
+                 cfg.evict_every, cfg.literal_return)
         h = C.c_void_p()
         rc = self.lib.crystalkv_create(C.byref(c), C.byref(h))
         if rc:
@@ -154,6 +159,16 @@ class CrystalKV:
         self._ck(self.lib.crystalkv_prefill(self._h, layer, _dev(k, (c.batch, P, c.n_kv_heads, c.head_dim)),
                                             _dev(v, (c.batch, P, c.n_kv_heads, c.head_dim)),
                                             _dev(q_last, (c.batch, c.n_q_heads, c.head_dim)), P, _stream()))
+
+    def prefill_window(self, layer, k, v, q_window, out_window=None):
+        c = self.cfg
+        P, W = k.shape[1], q_window.shape[0]
+        shape_q = (W, c.batch, c.n_q_heads, c.head_dim)
+        self._ck(self.lib.crystalkv_prefill_window(
+            self._h, layer, _dev(k, (c.batch, P, c.n_kv_heads, c.head_dim)),
+            _dev(v, (c.batch, P, c.n_kv_heads, c.head_dim)), _dev(q_window, shape_q), P, W,
+            None if out_window is None else _dev(out_window, shape_q), _stream()))
+        return out_window
 
     def decode_step(self, layer, q, k_new, v_new, out=None):
         c = self.cfg

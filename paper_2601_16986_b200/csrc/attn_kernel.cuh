@@ -584,7 +584,8 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
     int mine = 0, gmax = 0;
     for (int u = tid; u < U; u += NT) {
       const int uid = ((u / st.H) * st.L + p.layer) * st.H + (u % st.H);
-      const int n = p.n_in[uid];
+      int n = p.n_in[uid];
+      if (p.n_limit > 0) n = min(n, p.n_limit);   // a prompt token's causal view
       nin[u] = n;
       const int g = (n + p.append + GRP - 1) / GRP;
       mine += g;

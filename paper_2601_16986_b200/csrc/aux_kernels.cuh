@@ -9,11 +9,12 @@ namespace ckv {
 // ---------------------------------------------------------------------------------------
 // Prompt insertion for one layer: one CTA per (sequence, kv head).  Takes P + 1 slots from the
 // sequence's free list (P entries and the spare), copies the K/V rows into them and sets
-// pos = i, CRF = 0, tau = P - 1 (the time of the scoring pass that follows).
+// pos = i, CRF = 0 and tau = P - 1 (the time of the scoring pass that follows) or, when the
+// prompt's last tokens are replayed one by one, tau = i (the token's own arrival time).
 //   k, v: [batch][P][H][128] bf16
 __global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int* n_out, int layer,
                                                             const __nv_bfloat16* k,
-                                                            const __nv_bfloat16* v, int P) {
+                                                            const __nv_bfloat16* v, int P, int tau_is_pos) {
   __shared__ int s_top;
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
   const int uid = (seq * st.L + layer) * st.H + head;
@@ -34,12 +35,13 @@ __global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int* n_out
     if (tid == 0) n_out[uid] = 0;
     return;
   }
+  if (tid == 0) st.own[uid] = P + 1;
   const int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
   for (int i = tid; i <= P; i += NT) {
     st.list_slot[mb + i] = stack[top - 1 - i];
     if (i < P) {
       st.meta_pos[mb + i] = i;
-      st.meta_tau[mb + i] = P - 1;
+      st.meta_tau[mb + i] = tau_is_pos ? i : P - 1;
       st.meta_crf[mb + i] = 0.0f;
     }
   }
@@ -233,7 +235,7 @@ __global__ void __launch_bounds__(NT) shrink_kernel(State st, int* n_cur, int la
 
 // ---------------------------------------------------------------------------------------
 // Consistency check of slot ownership: every pool slot of a sequence must be owned exactly
-// once, either by the free list or by one head (its n entries and its spare).
+// once, either by the free list or by one head (its n entries and its spares).
 __global__ void mark_free_kernel(State st, int* seen) {
   const int seq = blockIdx.y;
   const int top = st.free_top[seq];
@@ -249,8 +251,9 @@ __global__ void mark_owned_kernel(State st, const int* n_cur, int layer, int* se
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
   const int uid = (seq * st.L + layer) * st.H + head;
   const size_t mb = (size_t)uid * st.cap;
-  const int n = n_cur[uid];
-  for (int i = threadIdx.x; i <= n; i += blockDim.x) {   // position n is the spare
+  const int own = st.own[uid];
+  if (threadIdx.x == 0 && own < n_cur[uid] + 1) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);   // no spare
+  for (int i = threadIdx.x; i < own; i += blockDim.x) {   // the entries, then the spares
     const int s = st.list_slot[mb + i];
     if (s < 0 || s >= st.slots_per_seq) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);
     else atomicAdd(&seen[(size_t)seq * st.slots_per_seq + s], 1);

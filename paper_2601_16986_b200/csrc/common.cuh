@@ -22,7 +22,7 @@ constexpr int NSETS = 16;           // logit scratch sets cycled by consecutive 
 
 // error word bits raised by device-side consistency checks (never a trap)
 constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence's free list was empty
-constexpr int ERR_OVER_EVICT = 2;       // a decode step found a head more than one entry over budget
+constexpr int ERR_OVER_EVICT = 2;       // a decode step found a head further over its budget than the eviction period allows
 constexpr int ERR_CAPACITY = 4;         // a head's list would outgrow its capacity
 constexpr int ERR_NUCLEUS = 8;          // the top-p threshold search did not find its boundary
 constexpr int ERR_COPY_TIMEOUT = 16;    // a bulk copy into shared memory did not complete within a second
@@ -40,6 +40,8 @@ struct State {
   float* meta_crf;   // [units][cap] CRF at tau
   int* nbuf[2];      // [2][units] entry counts, double buffered: a step reads one and writes the other
   int* budget;       // [units] == [batch][L][H]
+  int* own;          // [units] list positions [0, own) hold slots that belong to the head: its entries, then
+                     // its spares (one in steady state; up to the eviction period with a buffered cadence)
   const float* tab;  // lambda^D, D in [0, max_context]
   int* errword;
   unsigned long long* counters;  // entries attended, hits, evictions
@@ -76,6 +78,10 @@ struct DecodeParams {
   int release;    // 1: freed slots beyond one spare go back to the free list (no pops in this launch)
   int early;      // 1: the lists and rows of this layer are final, so the attention kernel may read them
                   //    before the kernel ahead of it in the stream has completed
+  int n_limit;    // > 0: only the first n_limit entries of every head take part (a prompt token's causal view)
+  int hold;       // 1: Algorithm 1 stops after step 3; lengths and lists stay as they are
+  int evict_every;   // m >= 1: step 4 waits until a head is m entries over its budget, then removes them all
+  int literal;    // 1: Algorithm 1 is skipped for a head below its budget (its first line as printed)
   float scale;    // logit scale
   float scale_log2;
   float top_p;
@@ -144,12 +150,13 @@ __device__ __forceinline__ int block_excl_scan(int v, int* red, int& total) {
   return base + inc - v;
 }
 
-// A head keeps its length and takes a fresh spare slot for list position n (decode steps in
-// which nothing left the head).  One thread calls it.
+// A head keeps its length and, unless it still owns a spare there, takes a fresh slot for list
+// position n (decode steps in which nothing left the head).  One thread calls it.
 __device__ __forceinline__ void keep_and_refill(const State& st, int* n_out, int uid, int seq, int n,
                                                 bool append) {
   n_out[uid] = n;
   if (!append) return;
+  if (st.own[uid] > n) return;   // one of the head's own spares is at list position n already
   if (n + 1 > st.cap) {
     atomicOr(st.errword, ERR_CAPACITY);
     return;
@@ -160,6 +167,7 @@ __device__ __forceinline__ void keep_and_refill(const State& st, int* n_out, int
     atomicOr(st.errword, ERR_FREE_UNDERFLOW);
   } else {
     st.list_slot[(size_t)uid * st.cap + n] = st.free_stack[(size_t)seq * st.slots_per_seq + idx];
+    st.own[uid] = n + 1;
   }
 }
 

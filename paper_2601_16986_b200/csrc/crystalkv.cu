@@ -163,6 +163,8 @@ int validate(const crystalkv_config_t* c, std::string& why) {
   if (c->lambda > 1.f) { why = "lambda above 1"; return CRYSTALKV_EINVAL; }
   if (c->sm_scale < 0.f) { why = "negative sm_scale"; return CRYSTALKV_EINVAL; }
   if (c->device < 0) { why = "negative device"; return CRYSTALKV_EINVAL; }
+  if (c->evict_every < 0 || c->evict_every > 4096) { why = "evict_every outside [0, 4096]"; return CRYSTALKV_EINVAL; }
+  if (c->literal_return != 0 && c->literal_return != 1) { why = "literal_return must be 0 or 1"; return CRYSTALKV_EINVAL; }
   return CRYSTALKV_OK;
 }
 
@@ -202,6 +204,8 @@ DecodeParams make_params(crystalkv_t* h, int layer, int set) {
   p.scale = h->cfg.sm_scale;
   p.scale_log2 = h->cfg.sm_scale * 1.44269504088896340736f;
   p.top_p = h->cfg.top_p;
+  p.evict_every = h->cfg.evict_every;
+  p.literal = h->cfg.literal_return;
   return p;
 }
 
@@ -315,16 +319,17 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   if (c.sm_scale == 0.f) c.sm_scale = (float)(1.0 / std::sqrt((double)c.head_dim));
   if (c.min_budget == 0) c.min_budget = std::min(c.budget_per_head, std::max(16, c.budget_per_head / 8));
   if (c.max_budget == 0) c.max_budget = 4 * c.budget_per_head;
+  if (c.evict_every < 1) c.evict_every = 1;
   const bool evict = c.mode == CRYSTALKV_MODE_EVICT;
   h->G = c.n_q_heads / c.n_kv_heads;
   h->U = c.batch * c.n_kv_heads;
   h->units = h->U * c.n_layers;
-  // list positions per head: entries up to the largest budget plus the arriving one and the
-  // answer-stage tail, plus the spare; FullKV keeps every token
-  h->cap = evict ? c.max_budget + 1 + c.max_answer_tokens + 1 : c.max_context + 1;
+  // list positions per head: entries up to the largest budget plus those that arrive before the
+  // next eviction and the answer-stage tail, plus the spare; FullKV keeps every token
+  h->cap = evict ? c.max_budget + c.evict_every + c.max_answer_tokens + 1 : c.max_context + 1;
   h->cap = (h->cap + GRP - 1) / GRP * GRP;   // whole 16-entry groups: a piece's slot ids are one aligned bulk copy
   h->slots_per_seq = (long long)c.n_layers * c.n_kv_heads *
-                     (evict ? (long long)c.budget_per_head + 1 + c.max_answer_tokens : (long long)c.max_context + 1);
+                     (evict ? (long long)c.budget_per_head + c.evict_every + c.max_answer_tokens : (long long)c.max_context + 1);
   if (h->slots_per_seq > 0x7fffffffLL) { g_create_err = "more than 2^31 slots per sequence"; delete h; return CRYSTALKV_EINVAL; }
 
 #define CREATE_FAIL(code_)                    \
@@ -382,6 +387,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   DA(&st.nbuf[0], h->units);
   DA(&st.nbuf[1], h->units);
   DA(&st.budget, h->units);
+  DA(&st.own, h->units);
   DA(&h->tab, (size_t)c.max_context + 1);
   st.tab = h->tab;
   DA(&st.errword, 1);
@@ -416,6 +422,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   fill_int_kernel<<<256, 256>>>(st.budget, h->units, c.budget_per_head);
   CKC(cudaMemset(st.nbuf[0], 0, (size_t)h->units * sizeof(int)));
   CKC(cudaMemset(st.nbuf[1], 0, (size_t)h->units * sizeof(int)));
+  CKC(cudaMemset(st.own, 0, (size_t)h->units * sizeof(int)));
   CKC(cudaMemset(st.errword, 0, sizeof(int)));
   CKC(cudaMemset(st.counters, 0, 4 * sizeof(unsigned long long)));
   CKC(cudaGetLastError());
@@ -446,11 +453,13 @@ int crystalkv_time(crystalkv_t* h, int layer) {
   return h->t_layer[layer];
 }
 
-int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v, const void* q_last,
-                      int P, void* stream) {
+// Prompt insertion and the Algorithm 1 passes that seed CRF/tau: one pass with the last query
+// (W = 0) or a replay of the last W queries, each over the tokens up to its own.
+static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* v, const void* q,
+                          int P, int W, void* out_window, void* stream) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
-  if (!k || !v || !q_last) return fail(h, CRYSTALKV_EINVAL, "null tensor");
+  if (!k || !v || !q) return fail(h, CRYSTALKV_EINVAL, "null tensor");
   const crystalkv_config_t& c = h->cfg;
   const bool evict = c.mode == CRYSTALKV_MODE_EVICT;
   if (P < 1) return fail(h, CRYSTALKV_EINVAL, "P must be >= 1");
@@ -464,24 +473,42 @@ int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v, c
   if (rc) return rc;
   prefill_insert_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer,
                                             static_cast<const __nv_bfloat16*>(k),
-                                            static_cast<const __nv_bfloat16*>(v), P);
+                                            static_cast<const __nv_bfloat16*>(v), P, W > 0 ? 1 : 0);
   CK(h, cudaGetLastError());
   if (evict) {
-    // one Algorithm 1 pass with Q^last at t = P-1: seeds CRF/tau, evicts down to the budget
-    DecodeParams p = make_params(h, layer, 0);
-    p.q = static_cast<const __nv_bfloat16*>(q_last);
-    p.k_new = p.v_new = nullptr;
-    p.out = h->dummy_out;
-    p.t = P - 1;
-    p.append = 0; p.track = 1; p.release = 1;
-    rc = launch_step(h, p, layer, s);
-    if (rc) return rc;
+    const int passes = W > 0 ? W : 1;
+    const size_t qn = (size_t)c.batch * c.n_q_heads * HD;
+    for (int i = 0; i < passes; ++i) {
+      // Algorithm 1 with the query of token t: steps 1-3 for every query, step 4 (down to the
+      // budget, freed slots back to the free list) after the last one
+      const int t = P - passes + i;
+      DecodeParams p = make_params(h, layer, 0);
+      p.q = static_cast<const __nv_bfloat16*>(q) + (size_t)i * qn;
+      p.k_new = p.v_new = nullptr;
+      p.out = out_window ? static_cast<__nv_bfloat16*>(out_window) + (size_t)i * qn : h->dummy_out;
+      p.t = t;
+      p.append = 0; p.track = 1; p.release = 1;
+      if (i < passes - 1) { p.n_limit = t + 1; p.hold = 1; }
+      rc = launch_step(h, p, layer, s);
+      if (rc) return rc;
+    }
     rc = join_side(h, s);
     if (rc) return rc;
     h->par[layer] ^= 1;
   }
   h->t_layer[layer] = P - 1;
   return CRYSTALKV_OK;
+}
+
+int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v, const void* q_last,
+                      int P, void* stream) {
+  return prefill_common(h, layer, k, v, q_last, P, 0, nullptr, stream);
+}
+
+int crystalkv_prefill_window(crystalkv_t* h, int layer, const void* k, const void* v,
+                             const void* q_window, int P, int W, void* out_window, void* stream) {
+  if (h && (W < 1 || W > P)) return fail(h, CRYSTALKV_EINVAL, "W must be in [1, P]");
+  return prefill_common(h, layer, k, v, q_window, P, W, out_window, stream);
 }
 
 int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* k_new,
@@ -798,7 +825,7 @@ int crystalkv_check(crystalkv_t* h, void* stream) {
   CK(h, cudaMemsetAsync(h->st.errword, 0, sizeof(int), s));
   std::string msg = "device error word:";
   if (w & ERR_FREE_UNDERFLOW) msg += " free-list underflow;";
-  if (w & ERR_OVER_EVICT) msg += " head more than one entry over budget in a decode step;";
+  if (w & ERR_OVER_EVICT) msg += " head further over its budget than the eviction period in a decode step;";
   if (w & ERR_CAPACITY) msg += " head list capacity exceeded;";
   if (w & ERR_NUCLEUS) msg += " top-p boundary not found;";
   if (w & ERR_COPY_TIMEOUT) msg += " a bulk copy into shared memory timed out;";

@@ -37,12 +37,12 @@ __device__ __forceinline__ void swap_into(const State& st, size_t mb, int dst, i
   st.list_slot[mb + src] = freed;
 }
 
-// Spares at list positions (n_new, n_old] return to the sequence's free list (the k freed
-// slots and the head's previous spare at n_old, minus the one at n_new that stays with the
-// head).  Only called from launches in which no head pops a slot.
-__device__ __forceinline__ void release_spares(const State& st, size_t mb, int seq, int n_new,
-                                               int n_old, int* s_base) {
-  const int cnt = n_old - n_new;
+// The head's spares beyond the one at list position n_new (the freed slots and the spares it
+// held before) return to the sequence's free list.  Only called from launches in which no head
+// pops a slot.
+__device__ __forceinline__ void release_spares(const State& st, size_t mb, int uid, int seq, int n_new,
+                                               int* s_base) {
+  const int cnt = st.own[uid] - (n_new + 1);
   if (cnt <= 0) return;
   if (threadIdx.x == 0) *s_base = atomicAdd(&st.free_top[seq], cnt);
   __syncthreads();
@@ -50,6 +50,7 @@ __device__ __forceinline__ void release_spares(const State& st, size_t mb, int s
   int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
   for (int r = threadIdx.x; r < cnt; r += NT) stack[base + r] = st.list_slot[mb + n_new + 1 + r];
   __syncthreads();
+  if (threadIdx.x == 0) st.own[uid] = n_new + 1;
 }
 
 // Removes the k lowest entries (1 <= k < n) of head `uid` at time t.  With `release` the head
@@ -137,7 +138,7 @@ __device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n,
     n_out[uid] = nk;
     atomicAdd(&st.counters[2], (unsigned long long)k);
   }
-  if (release) release_spares(st, mb, seq, nk, n, s_krem);
+  if (release) release_spares(st, mb, uid, seq, nk, s_krem);
 }
 
 }  // namespace ckv

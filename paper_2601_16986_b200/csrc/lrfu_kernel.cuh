@@ -378,7 +378,8 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   const unsigned long long w_theta = mass_of(__uint_as_float(theta));
 
   // ---- steps 2-3: CRF/tau update; step 4 candidates
-  const int k_evict = n - fr.budget;
+  // step 4 runs once the head is evict_every entries over its budget, and then for all of them
+  const int k_evict = (!p.hold && n - fr.budget >= p.evict_every) ? n - fr.budget : 0;
   uint32_t bk0 = 0xffffffffu, bk1 = 0xffffffffu, bk2 = 0xffffffffu;
   int bidx = -1, nhit = 0;
   auto update = [&](int i, float pm, int pos_i, int tau, float crf, float dec) {
@@ -495,12 +496,12 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
     n_after = n - 1;
   } else if (k_evict > 1) {
     __syncthreads();
-    if (p.append && tid == 0) atomicOr(st.errword, ERR_OVER_EVICT);
+    if (p.append && k_evict > p.evict_every && tid == 0) atomicOr(st.errword, ERR_OVER_EVICT);
     evict_many(st, p.n_out, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh.ev,
                reinterpret_cast<int*>(pbar));
     n_after = n - min(k_evict, n - 1);
   }
-  if (n_after == n && tid == 0) keep_and_refill(st, p.n_out, uid, seq, n, p.append != 0);
+  if (n_after == n && tid == 0 && !p.hold) keep_and_refill(st, p.n_out, uid, seq, n, p.append != 0);
 }
 
 template <int G>
@@ -511,7 +512,8 @@ __global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
   const int uid = (seq * st.L + p.layer) * st.H + head;
   // one batch of requests: the length, the budget, the softmax reference, and the logit rows the
   // common path needs (requested for a full thread's worth, clamped to the scratch)
-  const int n_raw = ld_i32(p.n_in + uid);
+  int n_raw = ld_i32(p.n_in + uid);
+  if (p.n_limit > 0) n_raw = min(n_raw, p.n_limit);
   Front<G> fr;
   fr.budget = ld_i32(st.budget + uid);
 #pragma unroll
@@ -530,7 +532,11 @@ __global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
   }
   const int n = n_raw + p.append;
   if (n <= 0) {
-    if (threadIdx.x == 0) p.n_out[uid] = 0;
+    if (threadIdx.x == 0 && !p.hold) p.n_out[uid] = 0;
+    return;
+  }
+  if (p.literal && n < fr.budget) {   // Algorithm 1's first line as printed: nothing runs below the budget
+    if (threadIdx.x == 0 && !p.hold) keep_and_refill(st, p.n_out, uid, seq, n, p.append != 0);
     return;
   }
   if (n <= FRONT * NT) lrfu_unit<G, FRONT>(p, u, uid, seq, n, sh, fr);

@@ -39,18 +39,20 @@ class Report:
 
 class LockStep:
     def __init__(self, wl: Workload, sample_seqs, mode=0, min_budget=0, max_budget=0,
-                 max_answer_tokens=0, device="cuda"):
+                 max_answer_tokens=0, device="cuda", evict_every=1, literal_return=0):
         self.wl, self.seqs, self.dev = wl, list(sample_seqs), device
         ctx = wl.prompt + wl.think_steps + wl.answer_steps + 2
         self.gpu = CrystalKV(Config(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
                                     batch=wl.batch, budget_per_head=wl.budget_per_head, max_context=ctx,
                                     min_budget=min_budget, max_budget=max_budget,
-                                    max_answer_tokens=max_answer_tokens, top_p=wl.top_p, lam=wl.lam, mode=mode))
+                                    max_answer_tokens=max_answer_tokens, top_p=wl.top_p, lam=wl.lam, mode=mode,
+                                    evict_every=evict_every, literal_return=literal_return))
         bph = wl.budget_per_head
         self.ora = Oracle(OracleConfig(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
                                        batch=len(self.seqs), budget_per_head=bph, max_context=ctx,
                                        min_budget=min_budget or min(bph, max(16, bph // 8)),
-                                       max_budget=max_budget or 4 * bph, top_p=wl.top_p, lam=wl.lam, mode=mode))
+                                       max_budget=max_budget or 4 * bph, top_p=wl.top_p, lam=wl.lam, mode=mode,
+                                       evict_every=evict_every, literal_return=literal_return))
         self.rep = Report()
         self.t = wl.prompt - 1
         self._tie_seen = 0
@@ -68,6 +70,20 @@ class LockStep:
             self.gpu.prefill(l, k, v, q)
             idx = torch.tensor(self.seqs, device=self.dev)
             self.ora.prefill(l, k[idx].cpu(), v[idx].cpu(), q[idx].cpu())
+        self.gpu.check()
+
+    def prefill_window(self, W):
+        """Prompt with the last W queries replayed; the window's attention outputs are compared too."""
+        wl = self.wl
+        idx = torch.tensor(self.seqs, device=self.dev)
+        for l in range(wl.n_layers):
+            k, v = wl.prompt_kv(l, device=self.dev)
+            q = wl.queries(l, list(range(wl.prompt - W, wl.prompt)), device=self.dev).transpose(0, 1).contiguous()
+            out = torch.zeros_like(q)
+            self.gpu.prefill_window(l, k, v, q, out)
+            ref = self.ora.prefill_window(l, k[idx].cpu(), v[idx].cpu(), q[:, idx].cpu())
+            err = float(np.abs(out[:, idx].float().cpu().numpy() - ref).max())
+            self.rep.max_out_err = max(self.rep.max_out_err, err)
         self.gpu.check()
 
     def step(self, compare_state=True, layers=None):

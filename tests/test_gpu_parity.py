@@ -294,6 +294,67 @@ def test_host_buffer_steps_match_device_steps():
 
 
 # ------------------------------------------------------------------ error paths on a live handle
+@pytest.mark.parametrize("W,prompt,budget", [(1, 83, 53), (8, 83, 53), (32, 200, 96), (40, 40, 64), (16, 300, 256)])
+def test_observation_window_prefill(W, prompt, budget):
+    """Algorithm 1 replayed over the last W prompt queries (causal views, steps 1-3 each, one
+    eviction after the last), then think steps; window outputs, state and ownership compared."""
+    wl = Workload(name=f"win{W}", seed=300 + W, n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3,
+                  prompt=prompt, think_steps=40, budget_per_head=budget, outlier="flat", outlier_frac=0.05)
+    ls = LockStep(wl, [0, 2], max_answer_tokens=max(64, prompt - budget + 8))
+    ls.prefill_window(W)
+    ls.compare()
+    ls.gpu.validate()
+    for h in range(2):
+        assert len(ls.gpu.get_retained(1, 2, h)) == min(prompt, budget)
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
+@pytest.mark.parametrize("m,literal,prompt,budget", [(8, 0, 83, 53), (16, 0, 40, 64), (3, 1, 30, 64), (1, 1, 83, 53),
+                                                     (64, 0, 300, 256)])
+def test_buffered_cadence_and_literal_return(m, literal, prompt, budget):
+    """Eviction once a head is m entries over its budget (m leave per call) and Algorithm 1's
+    early return as printed; head lengths cycle between B and B + m - 1."""
+    wl = Workload(name=f"cad{m}", seed=400 + m, n_layers=2, n_q_heads=8, n_kv_heads=2, batch=3,
+                  prompt=prompt, think_steps=3 * m + 60, budget_per_head=budget, outlier="flat", outlier_frac=0.05)
+    ls = LockStep(wl, [0, 2], max_answer_tokens=max(40, prompt - budget + 8), evict_every=m, literal_return=literal)
+    ls.prefill()
+    ls.compare()
+    sizes = set()
+    for s in range(wl.think_steps):
+        ls.step()
+        sizes.add(len(ls.gpu.get_retained(0, 0, 0)))
+        if s % 7 == 0:
+            ls.gpu.validate()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert max(sizes) == budget + m - 1 and budget in sizes
+    ls.close()
+
+
+def test_buffered_cadence_with_reallocation_and_answer_stage():
+    """The buffered heads through Algorithm 2 (shrinking releases every spare but one) and into
+    the answer stage (which uses up the spares a head still owns before it takes new slots)."""
+    wl = Workload(name="cadre", seed=77, n_layers=3, n_q_heads=8, n_kv_heads=2, batch=2, prompt=64,
+                  think_steps=100, answer_steps=12, budget_per_head=48, outlier="perhead", outlier_lo=0.01, outlier_hi=0.3)
+    ls = LockStep(wl, [0, 1], min_budget=8, max_answer_tokens=16, evict_every=6)
+    ls.prefill()
+    for s in range(wl.think_steps):
+        ls.step()
+        if (s + 1) % 25 == 0:
+            ls.rebudget()
+    ls.set_stage_answer()
+    for _ in range(wl.answer_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert ls.rep.budgets_compared > 0
+    ls.close()
+
+
 def test_call_order_errors():
     from paper_2601_16986_b200 import Config, CrystalKV, CrystalKVError
     kv = CrystalKV(Config(n_layers=2, n_q_heads=4, n_kv_heads=2, batch=1, budget_per_head=32, max_context=64))
