@@ -258,6 +258,106 @@ def sweep_cell(wl, batch, budget, fullkv, context, steps, warmup, dev):
     return row
 
 
+def policy_cell(wl, dev, steps, warmup, lam=None, top_p=None, evict_every=1, window=0, survival=True):
+    """One cell of the policy grid on the workload's shape: decode throughput after `warmup`
+    think steps, the hit fraction, and what the retained sets of sequence 0 look like."""
+    import numpy as np
+    from paper_2601_16986_b200 import Config, CrystalKV
+    lam = wl.lam if lam is None else lam
+    top_p = wl.top_p if top_p is None else top_p
+    L, B, Hq, H, d, P = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.prompt
+    total = warmup + steps
+    kv = CrystalKV(Config(n_layers=L, n_q_heads=Hq, n_kv_heads=H, batch=B, budget_per_head=wl.budget_per_head,
+                          max_context=P + total + 2, top_p=top_p, lam=lam, evict_every=evict_every))
+    stream = torch.cuda.current_stream()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    prefill_ms = 0.0
+    with torch.no_grad():
+        for l in range(L):
+            k, v = wl.prompt_kv(l, device=dev)
+            W = max(window, 1)
+            q = wl.queries(l, list(range(P - W, P)), device=dev).transpose(0, 1).contiguous()
+            torch.cuda.synchronize()
+            ev[0].record(stream)
+            if window:
+                kv.prefill_window(l, k, v, q)
+            else:
+                kv.prefill(l, k, v, q[0])
+            ev[1].record(stream)
+            torch.cuda.synchronize()
+            prefill_ms += ev[0].elapsed_time(ev[1])
+            del k, v
+        pos = torch.arange(P, P + total)
+        Q = torch.stack([wl.queries(l, pos, device=dev).transpose(0, 1) for l in range(L)], 1).contiguous()
+        K = torch.stack([wl.keys(l, pos, device=dev).transpose(0, 1) for l in range(L)], 1).contiguous()
+        V = torch.stack([wl.values(l, pos, device=dev).transpose(0, 1) for l in range(L)], 1).contiguous()
+        OUT = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=dev)
+    lib, h = kv.lib, kv._h
+    sp = C.c_void_p(stream.cuda_stream)
+    P_ = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
+
+    def run(n0, n1):
+        for s in range(n0, n1):
+            for l in range(L):
+                rc = lib.crystalkv_decode_step(h, l, P_(Q[s, l]), P_(K[s, l]), P_(V[s, l]), P_(OUT[l]), sp)
+                if rc:
+                    raise RuntimeError(f"decode_step failed: {rc}")
+    run(0, warmup)
+    torch.cuda.synchronize()
+    c0 = kv.get_counters()
+    ev[0].record(stream)
+    run(warmup, total)
+    lib.crystalkv_join(h, sp)
+    ev[1].record(stream)
+    torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[1]) / steps
+    c1 = kv.get_counters()
+    kv.check()
+    entries = (c1["entries_attended"] - c0["entries_attended"]) / steps
+    peak, _ = measured_peaks()
+    gbs = entries * 512 / (ms / 1000.0) / 1e9
+    row = {"lambda": lam, "top_p": top_p, "evict_every": evict_every, "window": window,
+           "prefill_ms_per_layer": prefill_ms / L, "ms_per_step": ms, "steps_per_s": 1000.0 / ms,
+           "frac_of_measured_hbm": gbs / peak,
+           "hit_fraction": (c1["hits"] - c0["hits"]) / max(c1["entries_attended"] - c0["entries_attended"], 1),
+           "evictions_per_step_per_head": (c1["evictions"] - c0["evictions"]) / steps / (B * L * H)}
+    if survival:   # the retained sets of sequence 0, every layer and head
+        t_now = P + total - 1
+        ages, n_prompt, n_all, sinks, out_kept, out_seen = [], 0, 0, 0, 0, 0
+        for l in range(L):
+            outl = wl.is_outlier(l, torch.arange(t_now + 1), seqs=[0])[0].numpy()   # [pos, H]
+            for hh in range(H):
+                r = kv.get_retained(l, 0, hh)
+                ages.append(t_now - r)
+                n_all += len(r); n_prompt += int((r < P).sum()); sinks += int(r[0] == 0)
+                out_kept += int(outl[r, hh].sum()); out_seen += int(outl[:, hh].sum())
+        ages = np.concatenate(ages)
+        row.update({"retained_prompt_fraction": n_prompt / n_all, "sink_kept_fraction": sinks / (L * H),
+                    "median_age": float(np.median(ages)), "recent64_fraction": float((ages < 64).mean()),
+                    "outliers_kept_of_seen": out_kept / max(out_seen, 1),
+                    "retained_of_seen": n_all / (L * H * (t_now + 1))})
+    kv.close()
+    del Q, K, V, OUT
+    torch.cuda.empty_cache()
+    return row
+
+
+def run_policy(args, wl):
+    """lambda x top-p grid (Section 6.4's ablation axes), the eviction period and the prefill window on
+    the workload's shape: throughput must not depend on the policy's parameters; one JSON line per cell."""
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    wl = wl.scaled(rebudget_every=0)
+    warm = max(args.warmup, 3)
+    for lam in (0.0, 0.3, 0.6, 0.9, 1.0):
+        for top_p in (0.5, 0.7, 0.9):
+            print(json.dumps(policy_cell(wl, dev, args.steps, warm, lam=lam, top_p=top_p)), flush=True)
+    for m in (4, 16, 64):
+        print(json.dumps(policy_cell(wl, dev, args.steps, warm, evict_every=m)), flush=True)
+    for W in (1, 8, 32):
+        print(json.dumps(policy_cell(wl, dev, args.steps, warm, window=W)), flush=True)
+
+
 def run_sweep(args):
     """The 14B-shape sweep: batch x per-head budget in steady state, and the full-cache baseline
     (every one of `context` tokens kept) of the same library; one JSON line per cell."""
@@ -287,6 +387,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="14B-shape sweep (batch x budget, steady state) against the full-cache baseline; one JSON line per cell")
+    ap.add_argument("--policy-sweep", action="store_true",
+                    help="lambda x top-p grid, eviction period and prefill window on the workload's shape; one JSON line per cell")
     ap.add_argument("--context", type=int, default=32768, help="tokens kept per head by the full-cache baseline of --sweep")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
@@ -298,6 +400,10 @@ def main():
         wl = wl.scaled(n_layers=args.layers)
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.policy_sweep:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        return run_policy(args, wl)
     if args.sweep:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")

@@ -54,7 +54,7 @@ __device__ __forceinline__ void release_spares(const State& st, size_t mb, int u
 }
 
 // Removes the k lowest entries (1 <= k < n) of head `uid` at time t.  With `release` the head
-// must own a spare at list position n (true between steps and after prompt insertion).  `sh` is >= 1.2 KB of
+// must own a spare at list position n (true between steps and after prompt insertion).  `sh` is >= 1.2 KB (300 ints) of
 // shared scratch, `tmp` a global int scratch of >= n words.  All NT threads call it.
 __device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n, int k, int t,
                            bool release, int* sh, int* tmp) {
@@ -64,12 +64,15 @@ __device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n,
   int* s_krem = sh + 259;
   int* red = sh + 260;        // NW + 1
   const int tid = threadIdx.x;
+  int* s_done = sh + 260 + NW + 1;
   if (tid < 3) s_kw[tid] = 0;
-  if (tid == 0) *s_krem = k;
+  if (tid == 0) { *s_krem = k; *s_done = 0; }
   __syncthreads();
-  // MSB-first radix select of the k-th smallest 96-bit key, 8 bits per pass
-  for (int word = 0; word < 3; ++word) {
-    for (int shift = 24; shift >= 0; shift -= 8) {
+  // MSB-first radix select of the k-th smallest 96-bit key, 8 bits per pass.  The search stops
+  // as soon as every entry that shares the prefix found so far is among the k lowest: the
+  // prefix followed by all ones then separates the same set as the k-th key itself.
+  for (int word = 0; word < 3 && !*s_done; ++word) {
+    for (int shift = 24; shift >= 0 && !*s_done; shift -= 8) {
       for (int b = tid; b < 256; b += NT) hist[b] = 0;
       __syncthreads();
       const uint32_t k0 = s_kw[0], k1 = s_kw[1], k2 = s_kw[2];
@@ -99,7 +102,13 @@ __device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n,
           for (int b = 0; b < 8; ++b) {
             const int c = hist[tid * 8 + b];
             if (cum + c >= krem) {
-              s_kw[word] = static_cast<int>(kw[word] | (static_cast<uint32_t>(tid * 8 + b) << shift));
+              uint32_t found = kw[word] | (static_cast<uint32_t>(tid * 8 + b) << shift);
+              if (krem - cum == c) {   // the whole bucket leaves
+                found |= (shift > 0) ? ((1u << shift) - 1u) : 0u;
+                for (int x = word + 1; x < 3; ++x) s_kw[x] = static_cast<int>(0xffffffffu);
+                *s_done = 1;
+              }
+              s_kw[word] = static_cast<int>(found);
               *s_krem = krem - cum;
               break;
             }

@@ -158,6 +158,16 @@ class Workload:
         scale = torch.where(pos == 0, torch.full_like(scale, 8.0), scale)
         return (k.to(torch.float32) * scale.unsqueeze(-1)).to(torch.bfloat16)
 
+    def is_outlier(self, layer: int, positions, seqs=None, device="cpu") -> torch.Tensor:
+        """bool [S, P, n_kv_heads]: which keys carry the x3 outlier scaling."""
+        seqs = list(range(self.batch) if seqs is None else seqs)
+        H = self.n_kv_heads
+        if self.outlier == "none":
+            return torch.zeros(len(seqs), len(positions), H, dtype=torch.bool, device=device)
+        ho = self._field(STREAM_OUTLIER, seqs, layer, H, positions, device)
+        thr = (self.outlier_fraction(layer, device) * 4294967296.0).to(torch.int64)
+        return ho < thr.view(1, 1, -1)
+
     # convenience wrappers with the shapes the library's calls take
     def prompt_kv(self, layer: int, seqs=None, device="cpu"):
         """(k, v), each [S, prompt, H, d]."""
