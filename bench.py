@@ -373,6 +373,32 @@ def run_sweep(args):
             print(json.dumps(row), flush=True)
 
 
+def run_throughput_table(args):
+    """The shape of the paper's throughput table (Section 6.3) on one GPU: the 8B model shape at
+    the 8K and 16K reasoning levels (9 350 and 18 700 tokens), full cache against a fixed budget of
+    1024 entries per head and against 10 % of the level (935 and 1 870), each at batch 1 and at the
+    largest batch that fits (100 GB of K/V rows, which leaves room for the prompt tensors; at most 256
+    sequences per handle)."""
+    wl = WORKLOADS["cfg3_llama8b"]
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    L, H = wl.n_layers, wl.n_kv_heads
+    for level in (9350, 18700):
+        per_seq_full = L * H * level * 512
+        rows = [("full cache", None, 1), ("full cache", None, min(256, int(100e9 // per_seq_full)))]
+        for name, budget in (("fixed-1024", 1024), (f"ratio-10%-{level // 10}", level // 10)):
+            per_seq = L * H * (budget + 1) * 512
+            rows += [(name, budget, 1), (name, budget, min(256, int(100e9 // per_seq)))]
+        for name, budget, batch in rows:
+            fullkv = budget is None
+            row = sweep_cell(wl, batch, budget or 1024, fullkv, level, 8 if fullkv else args.steps,
+                             3 if fullkv else max(args.warmup, 3), dev)
+            row.update({"level": level, "row": name, "concurrent_tokens": batch * level})
+            if row.get("status") == "ok":
+                row["tokens_per_s"] = row["steps_per_s"] * batch
+            print(json.dumps(row), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -387,6 +413,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="14B-shape sweep (batch x budget, steady state) against the full-cache baseline; one JSON line per cell")
+    ap.add_argument("--throughput-table", action="store_true",
+                    help="8B shape at the 8K and 16K levels: full cache against fixed and ratio budgets, batch 1 and largest batch")
     ap.add_argument("--policy-sweep", action="store_true",
                     help="lambda x top-p grid, eviction period and prefill window on the workload's shape; one JSON line per cell")
     ap.add_argument("--context", type=int, default=32768, help="tokens kept per head by the full-cache baseline of --sweep")
@@ -400,6 +428,10 @@ def main():
         wl = wl.scaled(n_layers=args.layers)
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.throughput_table:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        return run_throughput_table(args)
     if args.policy_sweep:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
