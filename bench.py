@@ -463,7 +463,8 @@ def main():
     L, B, Hq, H, d = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
     total = args.warmup + args.steps
     n_e2e = max(0, args.e2e_steps)
-    ctx = wl.prompt + total + n_e2e + 2
+    n_med = 32          # steps timed one by one, after the e2e steps, for the median
+    ctx = wl.prompt + total + n_e2e + n_med + 2
     kv = CrystalKV(Config(n_layers=L, n_q_heads=Hq, n_kv_heads=H, batch=B, budget_per_head=wl.budget_per_head,
                           max_context=ctx, top_p=wl.top_p, lam=wl.lam, device=local))
     with torch.no_grad():
@@ -472,7 +473,7 @@ def main():
             kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], seqs=seqs, device=dev)[:, 0].contiguous())
             del k, v
         # all step inputs resident in HBM before the timed region: [steps][L][batch][heads][d]
-        pos = torch.arange(wl.prompt, wl.prompt + total + n_e2e)
+        pos = torch.arange(wl.prompt, wl.prompt + total + n_e2e + n_med)
         Q = torch.empty(len(pos), L, B, Hq, d, dtype=torch.bfloat16, device=dev)
         K = torch.empty(len(pos), L, B, H, d, dtype=torch.bfloat16, device=dev)
         V = torch.empty(len(pos), L, B, H, d, dtype=torch.bfloat16, device=dev)
@@ -570,13 +571,17 @@ def main():
         hv = [[V[total + s, l].cpu().pin_memory() for l in range(L)] for s in range(n_e2e)]
         ho = [torch.empty(B, Hq, d, dtype=torch.bfloat16).pin_memory() for l in range(L)]
         hp = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
+        hqp = [[hp(t) for t in row] for row in hq]
+        hkp = [[hp(t) for t in row] for row in hk]
+        hvp = [[hp(t) for t in row] for row in hv]
+        hop = [hp(t) for t in ho]
         barrier()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.perf_counter()
         f0.record(stream)
         for s in range(n_e2e):
             for l in range(L):
-                rc = lib.crystalkv_decode_step_host(h, l, hp(hq[s][l]), hp(hk[s][l]), hp(hv[s][l]), hp(ho[l]), sp)
+                rc = lib.crystalkv_decode_step_host(h, l, hqp[s][l], hkp[s][l], hvp[s][l], hop[l], sp)
                 if rc:
                     raise RuntimeError(f"decode_step_host failed: {rc}")
             if every and (total + s + 1) % every == 0:
@@ -591,6 +596,18 @@ def main():
                "d2h_bytes_per_step": L * B * Hq * d * 2, "steps": n_e2e}
         kv.check()
 
+    # one event per step (kept out of the timed region above: an event between two launches stops
+    # the second kernel from starting early)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_med + 1)]
+    barrier()
+    marks[0].record(stream)
+    for i in range(n_med):
+        one_step(total + n_e2e + i, False)
+        marks[i + 1].record(stream)
+    barrier()
+    median_ms = statistics.median(marks[i].elapsed_time(marks[i + 1]) for i in range(n_med))
+    kv.check()
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v_cpu, threads, desc = oracle_sample(wl, layers=1, steps=4)
@@ -604,7 +621,7 @@ def main():
             "config": config_of(wl, world),
             "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches["n"],
             "roofline": roofline, "cpu_baseline": cpu,
-            "rebudget_ms_in_timed_region": ms_rb,
+            "rebudget_ms_in_timed_region": ms_rb, "median_ms_per_step": median_ms,
         }))
     kv.close()
     if world > 1:

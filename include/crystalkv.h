@@ -123,8 +123,10 @@ int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* 
                           const void* v_new, void* out, void* stream);
 
 /*
- * The same step with HOST buffers (page-locked for asynchronous copies).  The inputs are
- * copied up on one stream of the handle and `out` is copied down on another, both ordered
+ * The same step with HOST buffers (page-locked for asynchronous copies; pageable memory works
+ * but its copies block the host).  The inputs are brought up on one stream of the handle (by
+ * one small kernel that reads the page-locked buffers through their device mapping, else by
+ * three copies) and `out` is copied down on another, both ordered
  * against the step on `stream` by events, so the copies of one layer run beside the kernels
  * of others.  No host synchronisation.  `out_host` is complete once `stream` has passed a
  * later crystalkv_join (or any call that reads the cache state) and has been synchronised;

@@ -57,6 +57,26 @@ __global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int* n_out
 }
 
 // ---------------------------------------------------------------------------------------
+// Brings one step's q, k_new and v_new from page-locked host memory (read over the bus through
+// its device mapping, 16 bytes per thread) into the staging buffers: one launch instead of three
+// copies.  It runs in the caller's stream directly ahead of the step's attention kernel, both
+// launched with programmatic stream serialisation: this kernel lets the attention kernel start
+// at once, fetches while the attention kernel of the previous layer is still running, and only
+// then waits for that kernel, so that its own completion, which the attention kernel behind it
+// waits for, implies the completion of everything ahead.
+__global__ void __launch_bounds__(NT) stage_in_kernel(uint4* __restrict__ dq, uint4* __restrict__ dk,
+                                                      uint4* __restrict__ dv, const uint4* __restrict__ hq,
+                                                      const uint4* __restrict__ hk, const uint4* __restrict__ hv,
+                                                      int nq, int nk) {
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  const int i = blockIdx.x * NT + threadIdx.x;
+  if (i < nq) dq[i] = hq[i];
+  else if (i < nq + nk) dk[i - nq] = hk[i - nq];
+  else if (i < nq + 2 * nk) dv[i - nq - nk] = hv[i - nq - nk];
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------------
 // Algorithm 2 input: per head, the sum of CRF decayed to t_last over the retained entries,
 // each term truncated to 2^-32 fixed point so the sum does not depend on the order.
 __global__ void __launch_bounds__(NT) crf_sum_kernel(State st, const int* n_cur, int t_last,

@@ -59,6 +59,7 @@ struct crystalkv {
   __nv_bfloat16 *dq[HOST_RING] = {}, *dk[HOST_RING] = {}, *dv[HOST_RING] = {}, *dout[HOST_RING] = {};
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   cudaEvent_t evIn[HOST_RING] = {}, evUse[HOST_RING] = {}, evOut[HOST_RING] = {};
+  long long outJoined = -1;   // newest host step whose copy back the caller's stream has waited for
   long long nHost = 0;             // host-buffer steps so far
   __nv_bfloat16* dummy_out = nullptr;
   float* tab = nullptr;
@@ -550,19 +551,56 @@ int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host, co
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)c.batch * c.n_q_heads * HD * 2, kb = (size_t)c.batch * c.n_kv_heads * HD * 2;
   if (h->t_layer[layer] < 0) return fail(h, CRYSTALKV_ESTATE, "decode before prefill");
-  // Staging set j: its inputs go up on the copy-in stream (behind the attention kernel and the
-  // copy back that used the set HOST_RING steps ago), the caller's stream waits for them, runs
-  // the step, and the result comes down on the copy-out stream behind the attention kernel.
+  // Staging set j was last used HOST_RING host steps ago.  Page-locked inputs that the GPU can
+  // address are fetched by one small kernel in the caller's stream; anything else (pageable
+  // memory, 16-byte misalignment) goes up by three copies on the copy-in stream, for which the
+  // caller's stream then waits.  The result comes down on the copy-out stream behind the
+  // attention kernel.
   const int j = (int)(h->nHost % crystalkv::HOST_RING);
-  if (h->nHost >= crystalkv::HOST_RING) {
-    CK(h, cudaStreamWaitEvent(h->copy_in, h->evUse[j], 0));
-    CK(h, cudaStreamWaitEvent(h->copy_in, h->evOut[j], 0));
+  const void* dev_view[3] = {nullptr, nullptr, nullptr};
+  const void* host_in[3] = {q_host, k_new_host, v_new_host};
+  bool mapped = true;
+  for (int i = 0; i < 3 && mapped; ++i) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host_in[i]) != cudaSuccess) { cudaGetLastError(); mapped = false; break; }
+    mapped = at.type == cudaMemoryTypeHost && at.devicePointer != nullptr &&
+             (reinterpret_cast<uintptr_t>(at.devicePointer) & 15) == 0;
+    dev_view[i] = at.devicePointer;
   }
-  CK(h, cudaMemcpyAsync(h->dq[j], q_host, qb, cudaMemcpyHostToDevice, h->copy_in));
-  CK(h, cudaMemcpyAsync(h->dk[j], k_new_host, kb, cudaMemcpyHostToDevice, h->copy_in));
-  CK(h, cudaMemcpyAsync(h->dv[j], v_new_host, kb, cudaMemcpyHostToDevice, h->copy_in));
-  CK(h, cudaEventRecord(h->evIn[j], h->copy_in));
-  CK(h, cudaStreamWaitEvent(s, h->evIn[j], 0));
+  if (mapped) {
+    // The set's staged inputs were read by an attention kernel HOST_RING launches back in this
+    // stream, which is complete before this kernel may start.  Its result buffer must have been
+    // copied down as well; a wait in the caller's stream costs several microseconds, so one wait
+    // on a newer copy covers the next steps too.
+    const long long n = h->nHost;
+    if (n >= crystalkv::HOST_RING && n - crystalkv::HOST_RING > h->outJoined) {
+      const long long target = n - crystalkv::HOST_RING / 2;
+      CK(h, cudaStreamWaitEvent(s, h->evOut[target % crystalkv::HOST_RING], 0));
+      h->outJoined = target;
+    }
+    const int nq = (int)(qb / 16), nk = (int)(kb / 16);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((nq + 2 * nk + NT - 1) / NT);
+    lc.blockDim = dim3(NT);
+    lc.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    CK(h, cudaLaunchKernelEx(&lc, stage_in_kernel, reinterpret_cast<uint4*>(h->dq[j]), reinterpret_cast<uint4*>(h->dk[j]),
+                             reinterpret_cast<uint4*>(h->dv[j]), static_cast<const uint4*>(dev_view[0]),
+                             static_cast<const uint4*>(dev_view[1]), static_cast<const uint4*>(dev_view[2]), nq, nk));
+  } else {
+    // the copy back of the step that used the set before ran behind that step's attention
+    // kernel, so its event covers both
+    if (h->nHost >= crystalkv::HOST_RING) CK(h, cudaStreamWaitEvent(h->copy_in, h->evOut[j], 0));
+    CK(h, cudaMemcpyAsync(h->dq[j], q_host, qb, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaMemcpyAsync(h->dk[j], k_new_host, kb, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaMemcpyAsync(h->dv[j], v_new_host, kb, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaEventRecord(h->evIn[j], h->copy_in));
+    CK(h, cudaStreamWaitEvent(s, h->evIn[j], 0));
+  }
   rc = crystalkv_decode_step(h, layer, h->dq[j], h->dk[j], h->dv[j], h->dout[j], stream);
   if (rc) return rc;
   CK(h, cudaEventRecord(h->evUse[j], s));
