@@ -109,6 +109,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
   }
 }
 
+// Named barriers 1..NW: the warps that hold the pieces of one head meet there.
+__device__ __forceinline__ void bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;\n" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int nthreads) {
+  asm volatile("bar.arrive %0, %1;\n" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 constexpr int MAX_STAGES = 12;  // a warp's ring never grows beyond this
 constexpr int PIECE_SOFT = 24;  // groups a piece may grow to when that saves merge rounds
 constexpr float LAZY = 8.0f;   // the running maximum (log2 domain) may trail the true one by this much
@@ -187,7 +195,8 @@ __device__ __forceinline__ void merge_small(const float* pbase, int PS, int npie
 // warp, ids requested through registers two fires ahead.
 template <bool DEEP>
 __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned char* smem, const int* off, const int* nin,
-                                              int U, int Ptot, int nWarps, int nall_rt, bool dyn, int pi, uint32_t bars_u32) {
+                                              int U, int Ptot, int nWarps, int nall_rt, bool dyn, int pi, uint32_t bars_u32,
+                                              int chunk0) {
   const State& st = p.st;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
   const int G = p.G;
@@ -231,6 +240,9 @@ __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned ch
     const int g_u = (n_tot + GRP - 1) / GRP;
     const int piece = pi - off[u], npieces = off[u + 1] - off[u];
     const int lo = (int)((long long)g_u * piece / npieces), hi = (int)((long long)g_u * (piece + 1) / npieces);
+    // A head whose pieces all belong to this CTA is merged through shared memory.
+    const int first_w = off[u] - chunk0;   // warp that streams the head's first piece
+    const bool local = !DEEP && chunk0 >= 0 && npieces > 1 && first_w >= 0 && first_w + npieces <= NW;
     const size_t mb = (size_t)uid * st.cap;
     const int* list = st.list_slot + mb;
     const unsigned char* pool = st.pool + (size_t)seq * st.slots_per_seq * SLOT_BYTES;
@@ -325,6 +337,7 @@ __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned ch
         if (lane == 0) atomicOr(st.errword, ERR_COPY_TIMEOUT);
         for (int s = 0; s < nst; ++s)
           if (s != csi) mbar_wait_bounded(bar0 + s * 8, (phases >> s) & 1u);
+        if (local) bar_arrive(1 + first_w, 32 * npieces);   // the head's other warps must not wait for this one
         return;
       }
       phases ^= 1u << csi;
@@ -437,6 +450,71 @@ __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned ch
         if (h1 < G) { p.sc.mfin[u * (2 * QH) + h1] = m1; p.sc.mfin[u * (2 * QH) + QH + h1] = ls1; }
       }
       if (lane == 0) {
+        atomicAdd(&st.counters[0], (unsigned long long)n_tot);
+        if (!p.track) keep_and_refill(st, p.n_out, uid, seq, n_tot, p.append != 0);
+      }
+      continue;
+    }
+    if (local) {
+      // ---- the piece's partial goes into this warp's ring (idle by now: every copy that was
+      // fired has been consumed); after a barrier of the head's warps each of them merges a
+      // share of the query heads from all the partials
+      constexpr int HS = HD + 4;   // row stride that spreads the four head pairs of a store over the banks
+      constexpr int WSTRIDE = STAGES * STAGE_BYTES;
+      float* mine = reinterpret_cast<float*>(smem + w * WSTRIDE);
+      float ls0 = l0, ls1 = l1;
+#pragma unroll
+      for (int x = 4; x < 32; x <<= 1) {
+        ls0 += __shfl_xor_sync(0xffffffffu, ls0, x);
+        ls1 += __shfl_xor_sync(0xffffffffu, ls1, x);
+      }
+      if (gid == 0) {
+        *reinterpret_cast<float2*>(mine + 2 * tig) = make_float2(m0, m1);
+        *reinterpret_cast<float2*>(mine + 8 + 2 * tig) = make_float2(ls0, ls1);
+      }
+      {
+        const int h0 = 2 * tig, h1 = 2 * tig + 1;
+        float* po = mine + 16 + gid;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          if (h0 < G) { po[h0 * HS + 16 * mt] = o[mt][0]; po[h0 * HS + 16 * mt + 8] = o[mt][2]; }
+          if (h1 < G) { po[h1 * HS + 16 * mt] = o[mt][1]; po[h1 * HS + 16 * mt + 8] = o[mt][3]; }
+        }
+      }
+      bar_sync(1 + first_w, 32 * npieces);
+      const unsigned char* base = smem + first_w * WSTRIDE;
+      for (int g = w - first_w; g < G; g += npieces) {
+        float pm[NW], pl[NW];
+        float4 v[NW];
+        float m = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < NW; ++j) {
+          const float* pp = reinterpret_cast<const float*>(base + (j < npieces ? j : 0) * WSTRIDE);
+          pm[j] = (j < npieces) ? pp[g] : -INFINITY;
+          pl[j] = (j < npieces) ? pp[8 + g] : 0.f;
+          v[j] = *reinterpret_cast<const float4*>(pp + 16 + g * HS + lane * 4);
+          m = fmaxf(m, pm[j]);
+        }
+        float L = 0.f;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < NW; ++j) {
+          const float c = (pm[j] > -INFINITY) ? ex2(pm[j] - m) : 0.f;
+          L = fmaf(pl[j], c, L);
+          a.x = fmaf(v[j].x, c, a.x); a.y = fmaf(v[j].y, c, a.y);
+          a.z = fmaf(v[j].z, c, a.z); a.w = fmaf(v[j].w, c, a.w);
+        }
+        const float iv = 1.0f / L;
+        uint2 pk;
+        pk.x = pack_bf16(a.x * iv, a.y * iv);
+        pk.y = pack_bf16(a.z * iv, a.w * iv);
+        *reinterpret_cast<uint2*>(p.out + ((size_t)(u * G + g)) * HD + lane * 4) = pk;
+        if (lane == 0 && p.track) {
+          p.sc.mfin[u * (2 * QH) + g] = m;
+          p.sc.mfin[u * (2 * QH) + QH + g] = L;
+        }
+      }
+      if (w == first_w && lane == 0) {
         atomicAdd(&st.counters[0], (unsigned long long)n_tot);
         if (!p.track) keep_and_refill(st, p.n_out, uid, seq, n_tot, p.append != 0);
       }
@@ -641,8 +719,15 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
     atomicExch(p.piece_ctr + (p.parity ^ 1), 0);
     __threadfence();
   }
-  int pi;
-  if (dyn) {
+  int pi, chunk0 = -1;
+  if (dyn && nall == STAGES) {
+    // A CTA takes NW consecutive pieces at once, so that most heads have all their pieces in one
+    // CTA and merge through shared memory.  There are at most as many such chunks as CTAs.
+    if (tid == 0) s_red[0] = atomicAdd(p.piece_ctr + p.parity, 1);
+    __syncthreads();
+    chunk0 = s_red[0] * NW;
+    pi = chunk0 + w;
+  } else if (dyn) {
     pi = 0;
     if (lane == 0) pi = atomicAdd(p.piece_ctr + p.parity, 1);
     pi = __shfl_sync(0xffffffffu, pi, 0);
@@ -651,8 +736,8 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   }
   if (pi >= Ptot) return;
 
-  if (nall > STAGES) stream_pieces<true>(p, smem, off, nin, U, Ptot, nWarps, nall, dyn, pi, bars_u32);
-  else stream_pieces<false>(p, smem, off, nin, U, Ptot, nWarps, nall, dyn, pi, bars_u32);
+  if (nall > STAGES) stream_pieces<true>(p, smem, off, nin, U, Ptot, nWarps, nall, dyn, pi, bars_u32, -1);
+  else stream_pieces<false>(p, smem, off, nin, U, Ptot, nWarps, nall, dyn, pi, bars_u32, chunk0);
 }
 
 }  // namespace ckv
