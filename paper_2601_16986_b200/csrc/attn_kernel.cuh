@@ -652,6 +652,20 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   const int G = p.G;
   const int PS = 16 + G * HD;
 
+  // This CTA's turn among the launch's CTAs, asked for now so that the answer is there when the
+  // split is known (used when CTAs take whole chunks of pieces).
+  // The counters of the other parity are cleared for the next launch: every take of the launch
+  // before this one happened before it let this one start, and the next launch cannot start
+  // before this CTA has passed the point where it lets it.
+  __shared__ int s_turn;
+  if (threadIdx.x == 0) {
+    s_turn = atomicAdd(p.piece_ctr + 2 + p.parity, 1);
+    if (blockIdx.x == 0) {
+      atomicExch(p.piece_ctr + (p.parity ^ 1), 0);
+      atomicExch(p.piece_ctr + 2 + (p.parity ^ 1), 0);
+      __threadfence();
+    }
+  }
   if (threadIdx.x < NW * STAGES + NW) mbar_init(bars_u32 + threadIdx.x * 8, 1);
   asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");   // made visible to the copy engine
   // ---- every CTA derives the same split.  T = groups a piece may hold at most, chosen so that
@@ -703,9 +717,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   const int Ptot = off[U];
   // Which piece a warp takes.  When every warp gets at most one, pieces go to the warps in the
   // order in which they become ready (one atomic each): CTAs that reach an SM late, because the
-  // kernel ahead held it longer, then find the pieces gone instead of finishing last.  The
-  // counter of the other parity is cleared for the next launch: all takes of the launch before
-  // this one happened before it let this one start.
+  // kernel ahead held it longer, then find the pieces gone instead of finishing last.
   // apc = pieces a CTA gets at most; its warps with a piece share the CTA's ring stages
   const int apc = min(NW, (Ptot + (int)gridDim.x - 1) / (int)gridDim.x);
   // A warp with four stages or more gives the last one to the slot ids of its piece (one bulk
@@ -715,17 +727,11 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   const int nall = apc <= 2 ? min(MAX_STAGES + 1, (NW * STAGES) / apc) : STAGES;
   const bool dyn = Ptot <= nWarps;
   if (dyn && nall > STAGES && w >= apc) return;   // a deep ring: the CTA's stages are shared out among its first apc warps
-  if (blockIdx.x == 0 && tid == 0) {
-    atomicExch(p.piece_ctr + (p.parity ^ 1), 0);
-    __threadfence();
-  }
   int pi, chunk0 = -1;
   if (dyn && nall == STAGES) {
     // A CTA takes NW consecutive pieces at once, so that most heads have all their pieces in one
     // CTA and merge through shared memory.  There are at most as many such chunks as CTAs.
-    if (tid == 0) s_red[0] = atomicAdd(p.piece_ctr + p.parity, 1);
-    __syncthreads();
-    chunk0 = s_red[0] * NW;
+    chunk0 = s_turn * NW;   // written before the barriers of the split
     pi = chunk0 + w;
   } else if (dyn) {
     pi = 0;

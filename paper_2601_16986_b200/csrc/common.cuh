@@ -66,7 +66,7 @@ struct DecodeParams {
   const __nv_bfloat16* k_new;   // [batch][H][128]
   const __nv_bfloat16* v_new;
   __nv_bfloat16* out;           // [batch][Hq][128]
-  int* piece_ctr;    // two counters (by launch parity) from which the attention warps take their pieces
+  int* piece_ctr;    // counters by launch parity: [0..1] the attention warps take pieces, [2..3] its CTAs take chunks of pieces
   int parity;
   const int* n_in;   // entry counts before this step
   int* n_out;        // entry counts after it

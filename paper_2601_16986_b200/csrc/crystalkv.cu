@@ -407,8 +407,8 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     CKC(cudaMemset(h->sc_ticket[i], 0, (size_t)h->U * sizeof(int)));
   }
   DA(&h->sc_pbar, (size_t)h->U * h->cap_s);
-  DA(&h->piece_ctr, 2);
-  CKC(cudaMemset(h->piece_ctr, 0, 2 * sizeof(int)));
+  DA(&h->piece_ctr, 4);
+  CKC(cudaMemset(h->piece_ctr, 0, 4 * sizeof(int)));
   const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
   for (int i = 0; i < crystalkv::HOST_RING; ++i) { DA(&h->dq[i], qn); DA(&h->dout[i], qn); DA(&h->dk[i], kn); DA(&h->dv[i], kn); }
   DA(&h->dummy_out, qn);
