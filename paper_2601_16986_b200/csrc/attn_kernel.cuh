@@ -239,7 +239,9 @@ __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned ch
     const int n_old = nin[u], n_tot = n_old + p.append;
     const int g_u = (n_tot + GRP - 1) / GRP;
     const int piece = pi - off[u], npieces = off[u + 1] - off[u];
-    const int lo = (int)((long long)g_u * piece / npieces), hi = (int)((long long)g_u * (piece + 1) / npieces);
+    // (32-bit products: g_u * npieces stays below 2^32 for any list that fits the pool)
+    const int lo = (int)((unsigned)g_u * (unsigned)piece / (unsigned)npieces);
+    const int hi = (int)((unsigned)g_u * (unsigned)(piece + 1) / (unsigned)npieces);
     // A head whose pieces all belong to this CTA is merged through shared memory.
     const int first_w = off[u] - chunk0;   // warp that streams the head's first piece
     const bool local = !DEEP && chunk0 >= 0 && npieces > 1 && first_w >= 0 && first_w + npieces <= NW;
@@ -679,6 +681,10 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
       int n = p.n_in[uid];
       if (p.n_limit > 0) n = min(n, p.n_limit);   // a prompt token's causal view
       nin[u] = n;
+      if (u % (int)gridDim.x == (int)blockIdx.x) {   // the head's slot list is asked into L2 now (each head by one CTA): the split below takes as long as the fetch
+        const char* row = reinterpret_cast<const char*>(st.list_slot + (size_t)uid * st.cap);
+        for (int b = 0; b < (n + 1) * 4; b += 128) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(row + b));
+      }
       const int g = (n + p.append + GRP - 1) / GRP;
       mine += g;
       gmax = max(gmax, g);
