@@ -651,8 +651,6 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
   __shared__ int s_red[NW + 1];
   __shared__ int s_mx[NW];
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-  const int G = p.G;
-  const int PS = 16 + G * HD;
 
   // This CTA's turn among the launch's CTAs, asked for now so that the answer is there when the
   // split is known (used when CTAs take whole chunks of pieces).

@@ -234,6 +234,23 @@ def test_more_heads_than_warps_in_the_grid():
     ls.close()
 
 
+@pytest.mark.parametrize("G", [1, 2, 3, 6, 7, 8])
+def test_large_launch_merges_inside_the_cta_for_every_group_size(G):
+    """A launch large enough that CTAs take eight pieces at once: three pieces per head, so some
+    heads lie inside one CTA (merged through shared memory) and some straddle two (merged through
+    global memory), for group sizes other than those of the named shapes."""
+    wl = Workload(name=f"big{G}", seed=500 + G, n_layers=1, n_q_heads=8 * G, n_kv_heads=8, batch=40,
+                  prompt=600, think_steps=24, budget_per_head=600, outlier="flat", outlier_frac=0.03)
+    ls = LockStep(wl, [0, 17, 39])
+    ls.prefill()
+    ls.compare()
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
 def test_very_long_heads_use_the_general_lrfu_path():
     """A head above 17 x 256 entries: the LRFU kernel keeps pbar in global scratch, the attention
     kernel cuts the head into many pieces (merge in several rounds)."""
