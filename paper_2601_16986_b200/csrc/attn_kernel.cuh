@@ -698,11 +698,12 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {
     // (Pieces are not made longer than that on purpose: issuing the 16 bulk copies of a group
     // blocks the issuing warp for about half a microsecond, as long as the group's MMAs take, so
     // the copy rate of a launch grows with the number of warps that stream.)
-    // Small launches (under eight groups per warp): pieces of up to PIECE_SOFT groups keep a unit at
-    // four pieces or fewer, which the merge handles in a single round of loads.  Large launches
-    // only keep the longest unit at eight pieces (one CTA's warps): there every warp that does
-    // not stream costs bandwidth, and longer pieces for all would idle a third of them.
-    T = max(T, min(PIECE_SOFT, (Gtot < 8 * nWarps) ? (gmax + 3) / 4 : (gmax + 7) / 8));
+    // Small launches would be cut into pieces of GMIN groups by the bound above.  Pieces of up to
+    // PIECE_SOFT groups keep the longest unit at eight pieces, which one CTA's warps stream and merge
+    // through shared memory (four pieces for units under 64 groups: shorter pieces than eight
+    // groups cost more in starts than they gain in parallel streams).  Large launches are not
+    // lengthened beyond that either: there every warp that does not stream costs bandwidth.
+    T = max(T, min(PIECE_SOFT, gmax >= 64 ? (gmax + 7) / 8 : (gmax + 3) / 4));
     T = max(T, GMIN);
     int run = 0;
     for (int b0 = 0; b0 < U; b0 += NT) {
