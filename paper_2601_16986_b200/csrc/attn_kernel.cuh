@@ -414,11 +414,14 @@ __device__ __forceinline__ void stream_pieces(const DecodeParams& p, unsigned ch
       {
         const uint32_t va = stage + vb;
 #pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-          uint32_t a[4];
+        for (int mt = 0; mt < 8; mt += 2) {   // two tiles at a time: the two MMAs of a tile depend on each other
+          uint32_t a[4], a2[4];
           ldsm_x4_t(a, va + mt * 32);
+          ldsm_x4_t(a2, va + mt * 32 + 32);
           mma_bf16(o[mt], a, b0, b1);
+          mma_bf16(o[mt + 1], a2, b0, b1);
           mma_bf16(o[mt], a, rr0, rr1);
+          mma_bf16(o[mt + 1], a2, rr0, rr1);
         }
       }
       csi = (csi + 1 == nst) ? 0 : csi + 1;
