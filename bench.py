@@ -559,7 +559,7 @@ def main():
                 "entries_per_launch": entries / n_launch, "hit_fraction": hits / max(entries, 1)}
     # DRAM traffic of one attn_kernel launch from the ncu capture summarised in
     # profiles/attn_lrfu_kernels_cfg4_qwen14b.md (same launch shape): read + write bytes per entry
-    NCU_DRAM_BYTES_PER_ENTRY = (135.13e6 + 2.07e6) / 262400.0   # caches left alone (--cache-control none), one pass
+    NCU_DRAM_BYTES_PER_ENTRY = (135.15e6 + 2.24e6) / 262400.0   # caches left alone (--cache-control none), one pass
     if wl.name == "cfg4_qwen14b" and not args.batch and not args.budget:
         roofline["traffic"] = NCU_DRAM_BYTES_PER_ENTRY * entries / n_launch
 
