@@ -251,6 +251,23 @@ def test_large_launch_merges_inside_the_cta_for_every_group_size(G):
     ls.close()
 
 
+def test_window_prefill_and_buffered_cadence_in_a_large_launch():
+    """The observation window's causal views and the eviction of several entries per call, in a
+    launch large enough that CTAs take eight pieces at once and merge in shared memory."""
+    wl = Workload(name="bigwin", seed=611, n_layers=1, n_q_heads=40, n_kv_heads=8, batch=40,
+                  prompt=640, think_steps=20, budget_per_head=600, outlier="perhead")
+    ls = LockStep(wl, [0, 21, 39], max_answer_tokens=64, evict_every=5)
+    ls.prefill_window(6)
+    ls.compare()
+    ls.gpu.validate()
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    assert len(ls.gpu.get_retained(0, 39, 7)) in range(600, 605)
+    ls.close()
+
+
 def test_very_long_heads_use_the_general_lrfu_path():
     """A head above 17 x 256 entries: the LRFU kernel keeps pbar in global scratch, the attention
     kernel cuts the head into many pieces (merge in several rounds)."""
