@@ -18,9 +18,14 @@
  * and a library scaled-dot-product attention; the hit mask against subset
  * enumeration; CRF against the closed form of Section 5.2 and the lambda = 0 / 1
  * limits; eviction against a full sort; Algorithm 2 against hand examples and its
- * invariants; "budget = entries per head" against Table 1's HBM-saving column; the
+ * invariants, the re-share after the cap against a second set of hand examples;
+ * "budget = entries per head" against Table 1's HBM-saving column; the
  * observation-window prefill, the buffered eviction cadence and the literal early
- * return against the same definition-level simulator as the plain trajectory.
+ * return against the same definition-level simulator as the plain trajectory; the
+ * shrink after a reallocation and after okv_set_budget against that simulator's
+ * ranking by the closed-form CRF at the time of the last step; the tie log against
+ * hand-built inputs on both sides of the window and against the conditions evaluated
+ * from the definitions along a run; export and import as a round trip.
  * Whole trajectories (which tokens survive thousands of steps) have no value printed
  * in the paper: parity unpinned for those beyond the per-step pins above.
  *

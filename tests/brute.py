@@ -72,6 +72,50 @@ class BruteUnit:
     def last(self, i):
         return self.hits[i][-1] if self.hits[i] else self.arrival[i]
 
+    def _drop(self, gone):
+        for name in ("pos", "K", "V", "hits", "arrival"):
+            setattr(self, name, [x for j, x in enumerate(getattr(self, name)) if j not in gone])
+
+    def shrink(self, budget, t_last):
+        """A budget that shrank (Algorithm 2, or set by hand): the head keeps its `budget` best
+        entries at once.  Ranking from the definitions: CRF is the Section 5.2 sum evaluated at
+        the time of the last step, then the last hit (or arrival) time, then the position; the
+        lowest leave.  Returns the smallest relative distance of the cut from flipping."""
+        self.B = budget
+        n, gap = len(self.pos), np.inf
+        if n > budget:
+            keys = sorted((self.crf(i, t_last), self.last(i), self.pos[i], i) for i in range(n))
+            kk = n - budget
+            a, b = keys[kk - 1][0], keys[kk][0]
+            if a != b:
+                gap = abs(b - a) / max(abs(a), abs(b))
+            self._drop({x[3] for x in keys[:kk]})
+        return gap
+
+    def tie_flags(self, q, t, eps):
+        """What the tie log should say about a think step at time t with query q, BEFORE the
+        step is taken: (nucleus, evict).  nucleus: the inclusive or the exclusive mass at the
+        last hit lies within eps (relative to p) of p, or the last hit's score is within eps
+        (relative to itself) of the first miss's.  evict: the k-th and (k+1)-th lowest CRF
+        differ by less than eps relative to the larger, without being equal."""
+        K = np.stack(self.K)
+        prob, _ = naive_attention(q, K, np.stack(self.V), self.scale)
+        pbar = prob.mean(axis=0)
+        S, _ = brute_hits(list(pbar), self.p)
+        srt = np.sort(pbar)[::-1]
+        c = np.cumsum(srt)
+        k = len(S)
+        nucleus = abs(c[k - 1] - self.p) / self.p < eps or abs((c[k - 2] if k > 1 else 0.0) - self.p) / self.p < eps
+        if k < len(srt) and srt[k - 1] > 0:
+            nucleus = nucleus or abs(srt[k - 1] - srt[k]) / srt[k - 1] < eps
+        evict = False
+        n = len(self.pos)
+        if n - self.B >= self.m:
+            crf = sorted(self.crf(i, t) + (1.0 if i in S else 0.0) for i in range(n))
+            a, b = crf[n - self.B - 1], crf[n - self.B]
+            evict = a != b and abs(b - a) < eps * max(abs(a), abs(b))
+        return bool(nucleus), bool(evict)
+
     def step(self, q, t, track=True, evict=True):
         """Attention at time t; returns (y, min_gap) where min_gap is the smallest
         relative distance of any decision from flipping (for skipping near-ties)."""
@@ -97,7 +141,5 @@ class BruteUnit:
                 a, b = keys[kk - 1][0], keys[kk][0]
                 if a != b:
                     gap = min(gap, abs(b - a) / max(abs(a), abs(b)))
-                gone = {x[3] for x in keys[:kk]}
-                for name in ("pos", "K", "V", "hits", "arrival"):
-                    setattr(self, name, [x for j, x in enumerate(getattr(self, name)) if j not in gone])
+                self._drop({x[3] for x in keys[:kk]})
         return y, gap
