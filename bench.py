@@ -58,6 +58,34 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def kernel_source_digest():
+    """sha256 over the CUDA sources: a traffic figure captured for other sources is not reported."""
+    import glob
+    import hashlib
+    hsh = hashlib.sha256()
+    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2601_16986_b200", "csrc", "*"))):
+        with open(path, "rb") as f:
+            hsh.update(f.read())
+    return hsh.hexdigest()[:16]
+
+
+def dram_traffic_from_profile(wl, args, entries_per_launch):
+    """DRAM bytes of one attention launch, scaled from the counters of an ncu capture of the same
+    launch shape (profiles/dram_traffic.json: bytes per entry, the workload and the digest of the
+    kernel sources it was taken with).  None when there is no capture for this workload or the
+    kernels have changed since."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    out = {"traffic": None, "traffic_source": "no capture for these kernel sources and this workload"}
+    if not os.path.exists(path) or args.batch or args.budget:
+        return out
+    with open(path) as f:
+        rec = json.load(f)
+    if rec.get("workload") != wl.name or rec.get("kernel_source_digest") != kernel_source_digest():
+        return out
+    return {"traffic": rec["dram_bytes_per_entry"] * entries_per_launch,
+            "traffic_source": "ncu capture of the same launch shape (profiles/dram_traffic.json), not this run"}
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons sampled every 200 ms while a region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -410,6 +438,9 @@ def main():
     ap.add_argument("--budget", type=int, default=0, help="override budget_per_head")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling a small case)")
     ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--prep", type=int, default=1024,
+                    help="untimed think steps (with their reallocations) before the warm-up, so that the timed steps see "
+                         "heads of unequal length; 0 times the state right after the prefill")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="14B-shape sweep (batch x budget, steady state) against the full-cache baseline; one JSON line per cell")
@@ -461,47 +492,78 @@ def main():
     # ranks differ only in the sequence ids their inputs are drawn for
     seqs = [rank * wl.batch + b for b in range(wl.batch)]
     L, B, Hq, H, d = wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
-    total = args.warmup + args.steps
+    every = wl.rebudget_every
     n_e2e = max(0, args.e2e_steps)
     n_med = 32          # steps timed one by one, after the e2e steps, for the median
-    ctx = wl.prompt + total + n_e2e + n_med + 2
+    # Phases, in steps after the prefill (global step index s; a reallocation follows every step
+    # with (s + 1) % rebudget_every == 0):
+    #   uniform  W + Ku steps in the fresh state (every head at the uniform budget): a second, best-case figure
+    #   prepare  untimed, until every head has filled and at least `--prep` steps with their
+    #            reallocations have run: the state the method lives in (heads of unequal length)
+    #   main     W warm-up steps, then the K timed steps; then the end-to-end and the median steps
+    n_uni = min(args.steps, 20) if args.prep else 0
+    s_uni = args.warmup + n_uni if n_uni else 0
+    s_prep = 0
+    if args.prep:
+        s_prep = max(args.prep, wl.budget_per_head - wl.prompt + 2 * max(every, 64))
+        if every:
+            s_prep = (s_prep + every - 1) // every * every
+        s_prep = max(s_prep, s_uni)
+    s_main = s_prep + args.warmup          # first timed step
+    s_end = s_main + args.steps
+    n_all = s_end + n_e2e + n_med
+    ctx = wl.prompt + n_all + 2
     kv = CrystalKV(Config(n_layers=L, n_q_heads=Hq, n_kv_heads=H, batch=B, budget_per_head=wl.budget_per_head,
                           max_context=ctx, top_p=wl.top_p, lam=wl.lam, device=local))
+    lib, h = kv.lib, kv._h
+    stream = torch.cuda.current_stream()
+    sp = C.c_void_p(stream.cuda_stream)
+
+    class StepInputs:
+        """q, k_new, v_new of `count` consecutive steps, resident in HBM: [steps][L][batch][heads][d]."""
+
+        def __init__(self, count):
+            self.count, self.first = count, None
+            self.Q = torch.empty(count, L, B, Hq, d, dtype=torch.bfloat16, device=dev)
+            self.K = torch.empty(count, L, B, H, d, dtype=torch.bfloat16, device=dev)
+            self.V = torch.empty(count, L, B, H, d, dtype=torch.bfloat16, device=dev)
+
+        def fill(self, first):
+            """Draws the inputs of steps first .. first + count - 1 (on the stream the steps run on)."""
+            with torch.no_grad():
+                for c0 in range(0, self.count, 64):
+                    n = min(64, self.count - c0)
+                    pp = torch.arange(wl.prompt + first + c0, wl.prompt + first + c0 + n)
+                    for l in range(L):
+                        self.Q[c0:c0 + n, l] = wl.queries(l, pp, seqs=seqs, device=dev).transpose(0, 1)
+                        self.K[c0:c0 + n, l] = wl.keys(l, pp, seqs=seqs, device=dev).transpose(0, 1)
+                        self.V[c0:c0 + n, l] = wl.values(l, pp, seqs=seqs, device=dev).transpose(0, 1)
+            self.first = first
+            self.qp = [[C.c_void_p(self.Q[i, l].data_ptr()) for l in range(L)] for i in range(self.count)]
+            self.kp = [[C.c_void_p(self.K[i, l].data_ptr()) for l in range(L)] for i in range(self.count)]
+            self.vp = [[C.c_void_p(self.V[i, l].data_ptr()) for l in range(L)] for i in range(self.count)]
+
+        def at(self, s):
+            if self.first is None or not (self.first <= s < self.first + self.count):
+                self.fill(s)
+            return s - self.first
+
     with torch.no_grad():
         for l in range(L):
             k, v = wl.prompt_kv(l, seqs=seqs, device=dev)
             kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], seqs=seqs, device=dev)[:, 0].contiguous())
             del k, v
-        # all step inputs resident in HBM before the timed region: [steps][L][batch][heads][d]
-        pos = torch.arange(wl.prompt, wl.prompt + total + n_e2e + n_med)
-        Q = torch.empty(len(pos), L, B, Hq, d, dtype=torch.bfloat16, device=dev)
-        K = torch.empty(len(pos), L, B, H, d, dtype=torch.bfloat16, device=dev)
-        V = torch.empty(len(pos), L, B, H, d, dtype=torch.bfloat16, device=dev)
-        chunk = 64
-        for l in range(L):
-            for c0 in range(0, len(pos), chunk):
-                pp = pos[c0:c0 + chunk]
-                Q[c0:c0 + len(pp), l] = wl.queries(l, pp, seqs=seqs, device=dev).transpose(0, 1)
-                K[c0:c0 + len(pp), l] = wl.keys(l, pp, seqs=seqs, device=dev).transpose(0, 1)
-                V[c0:c0 + len(pp), l] = wl.values(l, pp, seqs=seqs, device=dev).transpose(0, 1)
         OUT = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=dev)
     torch.cuda.synchronize()
     kv.check()
-
-    lib, h = kv.lib, kv._h
-    stream = torch.cuda.current_stream()
-    sp = C.c_void_p(stream.cuda_stream)
-    qp = [[C.c_void_p(Q[s, l].data_ptr()) for l in range(L)] for s in range(len(pos))]
-    kp = [[C.c_void_p(K[s, l].data_ptr()) for l in range(L)] for s in range(len(pos))]
-    vp = [[C.c_void_p(V[s, l].data_ptr()) for l in range(L)] for s in range(len(pos))]
     op = [C.c_void_p(OUT[l].data_ptr()) for l in range(L)]
-    every = wl.rebudget_every
     launches = {"n": 0}
     rb_events = []
 
-    def one_step(s, timed):
+    def one_step(s, inp, timed):
+        i = inp.at(s)
         for l in range(L):
-            rc = lib.crystalkv_decode_step(h, l, qp[s][l], kp[s][l], vp[s][l], op[l], sp)
+            rc = lib.crystalkv_decode_step(h, l, inp.qp[i][l], inp.kp[i][l], inp.vp[i][l], op[l], sp)
             if rc:
                 raise RuntimeError(f"decode_step failed: {rc}")
         if timed:
@@ -524,44 +586,76 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for s in range(args.warmup):
-        one_step(s, False)
-    barrier()
-    c0 = kv.get_counters()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clk:
+    peak, peak_kind = measured_peaks()
+
+    def timed_region(s0, s1, inp, sampler=None):
+        """Steps s0 .. s1 - 1 between two events; returns (ms, roofline figures of the region)."""
+        barrier()
+        c0 = kv.get_counters()
+        del rb_events[:]
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(stream)
-        for s in range(args.warmup, total):
-            one_step(s, True)
+        for s in range(s0, s1):
+            one_step(s, inp, True)
         lib.crystalkv_join(h, sp)       # the last layers' LRFU kernels are inside the timed region
         ev1.record(stream)
         barrier()
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
-    c1 = kv.get_counters()
-    kv.check()
-    ms_rb = sum(a.elapsed_time(b) for a, b in rb_events)
-    ms_per_step = ms_total / args.steps
-    value = world * args.steps / (ms_total / 1000.0)
-
-    # roofline of the dominant kernel (the fused decode kernel): algorithmic bytes per launch
-    n_launch = args.steps * L
-    entries = c1["entries_attended"] - c0["entries_attended"]
-    hits = c1["hits"] - c0["hits"]
-    io_bytes = n_launch * (2 * B * Hq * d * 2 + 2 * B * H * d * 2)
-    algo_bytes = entries * (512 + 4 + 8) + hits * 8 + io_bytes
-    kernel_ms = (ms_total - ms_rb) / n_launch
-    achieved = algo_bytes / n_launch / (kernel_ms / 1000.0) / 1e9
-    peak, peak_kind = measured_peaks()
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_kind": peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
+        ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+        c1 = kv.get_counters()
+        kv.check()
+        ms_rb = sum(a.elapsed_time(b) for a, b in rb_events)
+        # roofline of the dominant kernel (the attention kernel): algorithmic bytes per launch
+        n_launch = (s1 - s0) * L
+        entries = c1["entries_attended"] - c0["entries_attended"]
+        hits = c1["hits"] - c0["hits"]
+        io_bytes = n_launch * (2 * B * Hq * d * 2 + 2 * B * H * d * 2)
+        algo_bytes = entries * (512 + 4 + 8) + hits * 8 + io_bytes
+        kernel_ms = (ms_total - ms_rb) / n_launch
+        achieved = algo_bytes / n_launch / (kernel_ms / 1000.0) / 1e9
+        kv_only = entries * 512 / n_launch / (kernel_ms / 1000.0) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": peak_kind + " copy bandwidth of this pool's B200s",
+                "frac_of_nominal_8TBs": achieved / 8000.0,
+                "kv_rows_only": {"achieved": kv_only, "frac": kv_only / peak, "frac_of_nominal_8TBs": kv_only / 8000.0},
                 "kernel": "attn_kernel", "launch_us": kernel_ms * 1000.0,
                 "algorithmic_bytes_per_launch": algo_bytes / n_launch,
-                "entries_per_launch": entries / n_launch, "hit_fraction": hits / max(entries, 1)}
-    # DRAM traffic of one attn_kernel launch from the ncu capture summarised in
-    # profiles/attn_lrfu_kernels_cfg4_qwen14b.md (same launch shape): read + write bytes per entry
-    NCU_DRAM_BYTES_PER_ENTRY = (135.15e6 + 2.24e6) / 262400.0   # caches left alone (--cache-control none), one pass
-    if wl.name == "cfg4_qwen14b" and not args.batch and not args.budget:
-        roofline["traffic"] = NCU_DRAM_BYTES_PER_ENTRY * entries / n_launch
+                "entries_per_launch": entries / n_launch, "hit_fraction": hits / max(entries, 1),
+                "rebudgets_in_region": len(rb_events), "rebudget_ms_in_region": ms_rb}
+        return ms_total, roof
+
+    # ---- the fresh, uniform state (best case), then the untimed preparation
+    prep_in = StepInputs(64)
+    roofline_uniform = None
+    if n_uni:
+        for s in range(0, args.warmup):
+            one_step(s, prep_in, False)
+        prep_in.fill(args.warmup)          # the timed steps' inputs are resident before the region starts (Ku <= 20 < 64)
+        ms_u, roofline_uniform = timed_region(args.warmup, s_uni, prep_in)
+        roofline_uniform.update({"steps": n_uni, "ms_per_step": ms_u / n_uni, "value": world * n_uni / (ms_u / 1000.0),
+                                 "state": "fresh after the prefill: every head at the uniform budget"})
+    for s in range(s_uni, s_prep):
+        one_step(s, prep_in, False)
+    barrier()
+    kv.check()
+    del prep_in
+    budgets = kv.get_budgets()
+    state = {"steps_before_timed_region": s_main, "reallocations_before": (s_main // every) if every else 0,
+             "budget_min": int(budgets.min()), "budget_max": int(budgets.max())}
+
+    # ---- warm-up and the timed steps, inputs resident before the region starts
+    main_in = StepInputs(n_all - s_prep)
+    main_in.fill(s_prep)
+    barrier()
+    for s in range(s_prep, s_main):
+        one_step(s, main_in, False)
+    with ClockSampler(local) as clk:
+        ms_total, roofline = timed_region(s_main, s_end, main_in)
+    ms_rb = roofline["rebudget_ms_in_region"]
+    ms_per_step = ms_total / args.steps
+    value = world * args.steps / (ms_total / 1000.0)
+    roofline["state"] = "after the preparation: heads of unequal length" if s_prep else "as prefilled"
+    roofline.update(dram_traffic_from_profile(wl, args, roofline["entries_per_launch"]))
+    Q, K, V, total = main_in.Q, main_in.K, main_in.V, s_end - s_prep   # index of the first e2e step in the buffers
 
     # end to end: the same steps through the host-buffer entry point, copies inside the timed region
     e2e = None
@@ -584,7 +678,7 @@ def main():
                 rc = lib.crystalkv_decode_step_host(h, l, hqp[s][l], hkp[s][l], hvp[s][l], hop[l], sp)
                 if rc:
                     raise RuntimeError(f"decode_step_host failed: {rc}")
-            if every and (total + s + 1) % every == 0:
+            if every and (s_end + s + 1) % every == 0:
                 lib.crystalkv_rebudget(h, sp)
         lib.crystalkv_join(h, sp)
         f1.record(stream)
@@ -602,7 +696,7 @@ def main():
     barrier()
     marks[0].record(stream)
     for i in range(n_med):
-        one_step(total + n_e2e + i, False)
+        one_step(s_end + n_e2e + i, main_in, False)
         marks[i + 1].record(stream)
     barrier()
     median_ms = statistics.median(marks[i].elapsed_time(marks[i + 1]) for i in range(n_med))
@@ -610,17 +704,17 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v_cpu, threads, desc = oracle_sample(wl, layers=1, steps=4)
+        v_cpu, threads, desc = oracle_sample(wl, layers=min(L, 4), steps=16)
         cpu = {"value": v_cpu, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": config_of(wl, world),
+            "vs_baseline": None, "dtype": "bf16", "dtype_detail": "bf16 inputs and cache, bf16 tensor-core MMA, fp32 accumulate and softmax",
+            "data": "synthetic", "config": config_of(wl, world), "state": state,
             "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches["n"],
-            "roofline": roofline, "cpu_baseline": cpu,
+            "roofline": roofline, "roofline_uniform": roofline_uniform, "cpu_baseline": cpu,
             "rebudget_ms_in_timed_region": ms_rb, "median_ms_per_step": median_ms,
         }))
     kv.close()

@@ -216,19 +216,21 @@ int crystalkv_validate(crystalkv_t* h, void* stream);
  *
  * crystalkv_validate takes a temporary from cudaMalloc on every call.  That is not possible
  * where a framework has already claimed all device memory for its own pool (cudaMalloc then
- * fails although the framework has room), inside code that is being captured into a CUDA
- * graph in a mode that forbids allocation calls, or in a serving loop that may not take the
+ * fails although the framework has room), or in a serving loop that may not take the
  * device-wide synchronisation a cudaMalloc / cudaFree pair implies.  This entry point does the
  * same check with its per-slot counters in an array that is built into the library: it calls
- * no cudaMalloc, cudaFree or other allocating routine.
+ * no cudaMalloc, cudaFree or other allocating routine.  Like crystalkv_validate it copies its
+ * verdict to the host and synchronises `stream`, so it is not a call for a stream that is
+ * being captured.
  *
  *   counts_out_host  host int32[2] or NULL: [0] slot ids out of range, [1] slots not owned
  *                    exactly once (both 0 on a sound handle)
  *
  * Limits and rules
- *   - The array covers handles of at most 2^21 = 2 097 152 pool slots in total
- *     (batch * L * H * (budget_per_head + 1 + max_answer_tokens); 1 GiB of K/V rows).  A larger
- *     handle is refused with EINVAL and a message that says so; use crystalkv_validate there.
+ *   - The array covers handles of at most 2^21 = 2 097 152 pool slots in total (1 GiB of K/V
+ *     rows): batch * L * H * (budget_per_head + evict_every + max_answer_tokens) slots in evict
+ *     mode, batch * L * H * (max_context + 1) in FullKV mode.  A larger handle is refused with
+ *     EINVAL and a message that says so; use crystalkv_validate there.
  *   - Every GPU on which the library is loaded holds the array (8 MiB) until the process ends.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress,
  *     with that device made current).  Make that first call before any stream capture begins.

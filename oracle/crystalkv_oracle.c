@@ -212,8 +212,8 @@ static int nuc_cmp(const void *a, const void *b) {
  * last hit's score and the first miss's score.
  * Returns the number of hits.
  */
-int okv_hit_mask(const double *pbar, const int32_t *pos, int n, double p, uint8_t *hit,
-                 double rel_eps, int *near_tie) {
+static int hit_mask_ex(const double *pbar, const int32_t *pos, int n, double p, uint8_t *hit,
+                       double rel_eps, int *near_tie, int *last_hit, int *first_miss) {
     nuc_item *it = (nuc_item *)malloc((size_t)(n > 0 ? n : 1) * sizeof(nuc_item));
     for (int i = 0; i < n; ++i) { it[i].p = pbar[i]; it[i].pos = pos[i]; it[i].idx = i; hit[i] = 0; }
     qsort(it, (size_t)n, sizeof(nuc_item), nuc_cmp);
@@ -235,8 +235,16 @@ int okv_hit_mask(const double *pbar, const int32_t *pos, int n, double p, uint8_
             if (nh < n && last > 0.0 && fabs(last - it[nh].p) / last < rel_eps) *near_tie = 1;
         }
     }
+    /* the two entries on either side of the boundary, for the harness's flipped replays */
+    if (last_hit) *last_hit = nh > 0 ? it[nh - 1].idx : -1;
+    if (first_miss) *first_miss = nh < n ? it[nh].idx : -1;
     free(it);
     return nh;
+}
+
+int okv_hit_mask(const double *pbar, const int32_t *pos, int n, double p, uint8_t *hit,
+                 double rel_eps, int *near_tie) {
+    return hit_mask_ex(pbar, pos, n, p, hit, rel_eps, near_tie, NULL, NULL);
 }
 
 /* ------------------------------------------------------------------ Algorithm 1 steps 2-4 */
@@ -312,10 +320,12 @@ static int evict_lowest(okv_unit *u, const float *crf_temp, int k, double rel_ep
  * hold: steps 1-3 only (the observation-window replay of the prompt evicts once, at
  * its last query).
  * y (may be NULL): [G][d] fp32 attention output.
+ * flip (0 in every ordinary call): the harness's "what if the near-tie had gone the other
+ * way" replays move the hit boundary by one entry after the mask is taken: 1 = the first
+ * miss is a hit too, 2 = the last hit is a miss, 3 = those two trade places.
  */
-static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, int t,
-                      int track, int hold, float *y) {
-    okv_unit *u = unit_of(o, seq, layer, head);
+static void lrfu_pass_unit(okv *o, okv_unit *u, int seq, int layer, int head, const uint16_t *q, int t,
+                           int track, int hold, float *y, int flip) {
     int n = u->n, d = o->c.head_dim, G = o->c.n_q_heads / o->c.n_kv_heads;
     if (track && o->c.literal_return && n < u->budget) track = 0;
     const double **kr = (const double **)malloc((size_t)n * sizeof(void *));
@@ -339,17 +349,24 @@ static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, i
             pbar[i] = s / (double)G;
             pos[i] = u->e[i].pos;
         }
-        int near = 0;
-        okv_hit_mask(pbar, pos, n, (double)o->c.top_p, hit, o->c.tie_eps, &near);
-        if (near) log_tie(o, layer, seq, head, t, OKV_TIE_NUCLEUS);
+        int near = 0, last_hit = -1, first_miss = -1;
+        hit_mask_ex(pbar, pos, n, (double)o->c.top_p, hit, o->c.tie_eps, &near, &last_hit, &first_miss);
+        if (near && layer >= 0) log_tie(o, layer, seq, head, t, OKV_TIE_NUCLEUS);
+        if ((flip == 1 || flip == 3) && first_miss >= 0) hit[first_miss] = 1;
+        if ((flip == 2 || flip == 3) && last_hit >= 0) hit[last_hit] = 0;
         crf_update(o, u, t, hit, ct);
         int m = o->c.evict_every > 1 ? o->c.evict_every : 1;
         int over = n - u->budget;
-        if (!hold && over >= m && evict_lowest(u, ct, over, o->c.tie_eps))
+        if (!hold && over >= m && evict_lowest(u, ct, over, o->c.tie_eps) && layer >= 0)
             log_tie(o, layer, seq, head, t, OKV_TIE_EVICT);
         free(pbar); free(pos); free(hit); free(ct);
     }
     free(kr); free(vr); free(prob); free(yy);
+}
+
+static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, int t,
+                      int track, int hold, float *y) {
+    lrfu_pass_unit(o, unit_of(o, seq, layer, head), seq, layer, head, q, t, track, hold, y, 0);
 }
 
 /* ------------------------------------------------------------------ lifecycle */
@@ -714,6 +731,59 @@ int okv_import_state(okv *o, int layer, int seq, int head, const int32_t *rec, i
         unit_append(o, u, rec[3 * i], k + (size_t)i * d, v + (size_t)i * d, crf, rec[3 * i + 2]);
     }
     return OKV_OK;
+}
+
+/*
+ * Replays think-stage decode steps of ONE head outside the oracle's own state, for the
+ * harness: when the GPU's state differs from the oracle's after a logged near-tie, the
+ * difference is only forgiven if this replay, with the tie taken the other way, lands on the
+ * GPU's state exactly.  The head starts from n records (as okv_export_state writes them)
+ * with their K/V rows and a budget, then takes nsteps steps at times t_first, t_first+1, ..
+ * with the given queries [nsteps][G][d] and arriving rows [nsteps][d]; flips[s] is the flip
+ * of step s (see lrfu_pass_unit).  With append_first = 0 the first step appends nothing: it
+ * is the scoring pass of a prefill over the records given.  Uses the handle's configuration
+ * and decay table only; logs nothing.  Writes the final records (sorted by position) and returns their count, or the
+ * negated count if cap is too small.
+ */
+int okv_replay_unit(okv *o, const int32_t *rec, const uint16_t *k, const uint16_t *v, int n, int budget,
+                    int t_first, int append_first, int nsteps, const uint16_t *q, const uint16_t *k_new, const uint16_t *v_new,
+                    const int32_t *flips, int32_t *rec_out, int cap) {
+    int d = o->c.head_dim, G = o->c.n_q_heads / o->c.n_kv_heads;
+    okv_unit u;
+    memset(&u, 0, sizeof u);
+    u.budget = budget;
+    for (int i = 0; i < n; ++i) {
+        float crf;
+        uint32_t bits = (uint32_t)rec[3 * i + 1];
+        memcpy(&crf, &bits, 4);
+        unit_append(o, &u, rec[3 * i], k + (size_t)i * d, v + (size_t)i * d, crf, rec[3 * i + 2]);
+    }
+    for (int s = 0; s < nsteps; ++s) {
+        int t = t_first + s;
+        if (s > 0 || append_first) unit_append(o, &u, t, k_new + (size_t)s * d, v_new + (size_t)s * d, 0.0f, t);
+        lrfu_pass_unit(o, &u, 0, -1, 0, q + (size_t)s * G * d, t, 1, 0, NULL, flips ? flips[s] : 0);
+    }
+    int n_out = u.n;
+    if (n_out <= cap) {
+        int32_t *order = (int32_t *)malloc((size_t)(n_out ? n_out : 1) * sizeof(int32_t));
+        for (int i = 0; i < n_out; ++i) order[i] = i;
+        for (int i = 1; i < n_out; ++i) { /* insertion sort by position */
+            int32_t x = order[i];
+            int j = i - 1;
+            while (j >= 0 && u.e[order[j]].pos > u.e[x].pos) { order[j + 1] = order[j]; --j; }
+            order[j + 1] = x;
+        }
+        for (int i = 0; i < n_out; ++i) {
+            okv_entry *e = &u.e[order[i]];
+            uint32_t bits;
+            memcpy(&bits, &e->crf, 4);
+            rec_out[3 * i] = e->pos; rec_out[3 * i + 1] = (int32_t)bits; rec_out[3 * i + 2] = e->tau;
+        }
+        free(order);
+    }
+    for (int j = 0; j < u.n; ++j) { free(u.e[j].k); free(u.e[j].v); }
+    free(u.e);
+    return n_out <= cap ? n_out : -n_out;
 }
 
 int okv_tie_count(okv *o) { return o->n_ties; }

@@ -69,6 +69,7 @@ def _load():
         lib.okv_time.argtypes = [vp, i32]
         lib.okv_export_state.argtypes = [vp, i32, i32, i32, vp, i32]
         lib.okv_import_state.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp]
+        lib.okv_replay_unit.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32]
         lib.okv_tie_count.argtypes = [vp]
         lib.okv_get_ties.argtypes = [vp, vp, i32]
         lib.okv_clear_ties.argtypes = [vp]
@@ -219,6 +220,22 @@ class Oracle:
         rec = np.ascontiguousarray(rec, dtype=np.int32)
         kb, vb = _bits(k), _bits(v)
         self._lib.okv_import_state(self._h, layer, seq, head, _p(rec), len(rec), _p(kb), _p(vb))
+
+    def replay_unit(self, rec, k, v, budget, t_first, q, k_new, v_new, flips, append_first=True) -> np.ndarray:
+        """One head replayed outside the oracle's state from records rec [n,3] with rows k, v [n,d]:
+        len(flips) think steps at times t_first, t_first+1, .. with queries q [steps,G,d] and arriving
+        rows [steps,d], flips[s] moving the hit boundary of step s (0 none, 1 one hit more, 2 one
+        fewer, 3 swap).  append_first=False: the first step is a prefill's scoring pass (nothing
+        arrives).  -> final records [m,3] sorted by position."""
+        rec = np.ascontiguousarray(rec, dtype=np.int32)
+        flips = np.ascontiguousarray(flips, dtype=np.int32)
+        kb, vb, qb, knb, vnb = _bits(k), _bits(v), _bits(q), _bits(k_new), _bits(v_new)
+        cap = len(rec) + len(flips) + 1
+        out = np.zeros((cap, 3), dtype=np.int32)
+        n = self._lib.okv_replay_unit(self._h, _p(rec), _p(kb), _p(vb), len(rec), int(budget), int(t_first), int(bool(append_first)), len(flips),
+                                      _p(qb), _p(knb), _p(vnb), _p(flips), _p(out), cap)
+        assert n >= 0
+        return out[:n].copy()
 
     def ties(self) -> np.ndarray:
         """-> int32 [m,5] rows (layer, seq, head, t, kind)."""

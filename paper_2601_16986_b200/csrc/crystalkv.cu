@@ -11,10 +11,12 @@
 #include "../../include/crystalkv.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -71,20 +73,49 @@ struct crystalkv {
 namespace {
 
 thread_local std::string g_create_err;
+constexpr int MAX_DEVICES = 64;   // device ordinals this library keeps per-device state for
 
 int fail(crystalkv_t* h, int code, const std::string& msg) {
   if (h) h->err = msg;
   return code;
 }
 
+// An error that only says "not while this stream is being captured" leaves the context and the
+// handle intact; every other CUDA error is sticky for the handle.
+bool capture_refusal(cudaError_t e) {
+  return e >= cudaErrorStreamCaptureUnsupported && e <= cudaErrorStreamCaptureWrongThread;
+}
+
 #define CK(h, call)                                                                      \
   do {                                                                                   \
     cudaError_t e_ = (call);                                                             \
     if (e_ != cudaSuccess) {                                                             \
-      if (h) (h)->cuda_dead = true;                                                      \
+      if ((h) && !capture_refusal(e_)) (h)->cuda_dead = true;                            \
       return fail((h), CRYSTALKV_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
     }                                                                                    \
   } while (0)
+
+// Makes the handle's device current for the duration of a call and puts the caller's back.
+struct DeviceScope {
+  int prev = -1;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceScope(int dev) {
+    int cur = -1;
+    err = cudaGetDevice(&cur);
+    if (err == cudaSuccess && cur != dev) {
+      err = cudaSetDevice(dev);
+      if (err == cudaSuccess) prev = cur;
+    }
+  }
+  ~DeviceScope() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+  DeviceScope(const DeviceScope&) = delete;
+  DeviceScope& operator=(const DeviceScope&) = delete;
+};
+#define ON_DEVICE(h)                       \
+  DeviceScope dev_scope_((h)->cfg.device); \
+  CK((h), dev_scope_.err)
 
 template <typename T>
 int dalloc(crystalkv_t* h, T** p, size_t count) {
@@ -121,12 +152,17 @@ template <int G>
 cudaError_t launch_lrfu(const DecodeParams& p, int grid, cudaStream_t s) {
   // the same shared-memory carve-out as the attention kernel, so that CTAs of both can be
   // resident on one SM at the same time
-  static bool prepared = false;
-  if (!prepared) {
-    cudaError_t e = cudaFuncSetAttribute(lrfu_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                         (int)cudaSharedmemCarveoutMaxShared);
+  // (function attributes are kept per device)
+  static std::atomic<bool> prepared[MAX_DEVICES] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (!prepared[dev].load(std::memory_order_acquire)) {
+    e = cudaFuncSetAttribute(lrfu_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    prepared = true;
+    prepared[dev].store(true, std::memory_order_release);
   }
   lrfu_kernel<G><<<grid, NT, 0, s>>>(p);
   return cudaGetLastError();
@@ -163,7 +199,7 @@ int validate(const crystalkv_config_t* c, std::string& why) {
   if (c->top_p < 0.f || c->top_p > 1.f) { why = "top_p outside (0, 1]"; return CRYSTALKV_EINVAL; }
   if (c->lambda > 1.f) { why = "lambda above 1"; return CRYSTALKV_EINVAL; }
   if (c->sm_scale < 0.f) { why = "negative sm_scale"; return CRYSTALKV_EINVAL; }
-  if (c->device < 0) { why = "negative device"; return CRYSTALKV_EINVAL; }
+  if (c->device < 0 || c->device >= MAX_DEVICES) { why = "device ordinal outside [0, 64)"; return CRYSTALKV_EINVAL; }
   if (c->evict_every < 0 || c->evict_every > 4096) { why = "evict_every outside [0, 4096]"; return CRYSTALKV_EINVAL; }
   if (c->literal_return != 0 && c->literal_return != 1) { why = "literal_return must be 0 or 1"; return CRYSTALKV_EINVAL; }
   return CRYSTALKV_OK;
@@ -288,7 +324,7 @@ const char* crystalkv_last_error(crystalkv_t* h) { return h ? h->err.c_str() : g
 
 int crystalkv_destroy(crystalkv_t* h) {
   if (!h) return CRYSTALKV_OK;
-  cudaSetDevice(h->cfg.device);
+  DeviceScope scope(h->cfg.device);
   cudaDeviceSynchronize();
   if (h->side) cudaStreamDestroy(h->side);
   if (h->copy_in) cudaStreamDestroy(h->copy_in);
@@ -354,13 +390,17 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     if (r_) CREATE_FAIL(r_);                             \
   } while (0)
 
-  CKC(cudaSetDevice(c.device));
+  DeviceScope scope(c.device);
+  CKC(scope.err);
   cudaDeviceProp prop;
   CKC(cudaGetDeviceProperties(&prop, c.device));
   h->num_sms = prop.multiProcessorCount;
   h->smem = RING_BYTES + (NW * STAGES + NW) * 8 + (size_t)(2 * h->U + 1) * sizeof(int);
   int bps = 0;
-  CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem));
+  // The attribute belongs to the function, not to the handle: it is set to the most any handle
+  // can ask for, so that a later, smaller handle does not lower it under an earlier one.
+  const size_t smem_max = RING_BYTES + (NW * STAGES + NW) * 8 + (size_t)(2 * MAX_UNITS_PER_CALL + 1) * sizeof(int);
+  CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
   CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
   if (bps < 1) { h->err = "attention kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
   h->grid = h->num_sms * bps;
@@ -443,6 +483,7 @@ int crystalkv_set_stage(crystalkv_t* h, int stage) {
   if (stage != CRYSTALKV_STAGE_THINK && stage != CRYSTALKV_STAGE_ANSWER) return fail(h, CRYSTALKV_EINVAL, "bad stage");
   if (stage == CRYSTALKV_STAGE_THINK && h->answer_steps > 0)
     return fail(h, CRYSTALKV_ESTATE, "answer tokens were appended; the think stage cannot resume");
+  ON_DEVICE(h);
   if (stage != h->stage) CK(h, cudaStreamSynchronize(h->side));   // no LRFU kernel is left behind the switch
   h->prev_layer = -1;
   h->stage = stage;
@@ -468,7 +509,7 @@ static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* 
     return fail(h, CRYSTALKV_EINVAL, "prompt longer than budget_per_head + max_answer_tokens");
   if (P >= c.max_context) return fail(h, CRYSTALKV_EINVAL, "prompt reaches max_context");
   if (h->t_layer[layer] >= 0) return fail(h, CRYSTALKV_ESTATE, "layer already prefilled");
-  CK(h, cudaSetDevice(c.device));
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   rc = join_side(h, s);   // the insertion pops slots; no LRFU kernel may push or pop meanwhile
   if (rc) return rc;
@@ -520,6 +561,7 @@ int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* 
   const crystalkv_config_t& c = h->cfg;
   if (h->t_layer[layer] < 0) return fail(h, CRYSTALKV_ESTATE, "decode before prefill");
   const int t = h->t_layer[layer] + 1;
+  ON_DEVICE(h);
   if (t >= c.max_context) return fail(h, CRYSTALKV_ESTATE, "max_context reached");
   const bool track = c.mode == CRYSTALKV_MODE_EVICT && h->stage == CRYSTALKV_STAGE_THINK;
   if (c.mode == CRYSTALKV_MODE_EVICT && h->stage == CRYSTALKV_STAGE_ANSWER) {
@@ -547,6 +589,7 @@ int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host, co
   int rc = check_layer(h, layer);
   if (rc) return rc;
   if (!q_host || !k_new_host || !v_new_host || !out_host) return fail(h, CRYSTALKV_EINVAL, "null tensor");
+  ON_DEVICE(h);
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)c.batch * c.n_q_heads * HD * 2, kb = (size_t)c.batch * c.n_kv_heads * HD * 2;
@@ -616,6 +659,7 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
   const crystalkv_config_t& c = h->cfg;
   if (c.mode != CRYSTALKV_MODE_EVICT) return fail(h, CRYSTALKV_ESTATE, "rebudget in FullKV mode");
+  ON_DEVICE(h);
   const int t_last = h->t_layer[0], par = h->par[0];
   if (t_last < 0) return fail(h, CRYSTALKV_ESTATE, "rebudget before prefill");
   for (int l = 1; l < c.n_layers; ++l)
@@ -644,6 +688,7 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
   const crystalkv_config_t& c = h->cfg;
   if (c.mode != CRYSTALKV_MODE_EVICT) return fail(h, CRYSTALKV_ESTATE, "set_budget in FullKV mode");
   if (budget < 1 || budget > c.max_budget) return fail(h, CRYSTALKV_EINVAL, "budget outside [1, max_budget]");
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
@@ -659,6 +704,7 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
 
 int crystalkv_get_budgets(crystalkv_t* h, int32_t* out_host, void* stream) {
   if (!h || !out_host) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   CK(h, cudaMemcpyAsync(out_host, h->st.budget, (size_t)h->units * sizeof(int), cudaMemcpyDeviceToHost, s));
@@ -671,6 +717,7 @@ int crystalkv_export_state(crystalkv_t* h, int layer, int seq, int kv_head, int3
   int rc = check_unit(h, layer, seq, kv_head);
   if (rc) return rc;
   if (!host_buf || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  ON_DEVICE(h);
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
@@ -705,6 +752,7 @@ int crystalkv_get_retained(crystalkv_t* h, int layer, int seq, int kv_head, int3
   int rc = check_unit(h, layer, seq, kv_head);
   if (rc) return rc;
   if (!pos_out_host || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  ON_DEVICE(h);
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
@@ -725,6 +773,7 @@ int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head, cons
   int rc = check_unit(h, layer, seq, kv_head);
   if (rc) return rc;
   if (!host_buf || n_rec < 0) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  ON_DEVICE(h);
   const crystalkv_config_t& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
@@ -757,6 +806,7 @@ int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head, cons
 int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t* hits,
                            uint64_t* evictions, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   unsigned long long v[4];
@@ -774,6 +824,7 @@ int crystalkv_validate(crystalkv_t* h, void* stream) {
   const crystalkv_config_t& c = h->cfg;
   for (int l = 0; l < c.n_layers; ++l)
     if (h->t_layer[l] < 0) return fail(h, CRYSTALKV_ESTATE, "validate before every layer is prefilled");
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   const long long total = (long long)c.batch * h->slots_per_seq;
@@ -805,6 +856,7 @@ constexpr long long STATIC_SEEN_SLOTS = 1ll << 21;
 static __device__ __align__(256) int g_seen_static[STATIC_SEEN_SLOTS + 2];
 constexpr int STATIC_MAX_DEVICES = 64;
 static int* g_seen_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device ordinal
+static std::mutex g_seen_mu;                        // guards the look-up above
 
 int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
@@ -818,15 +870,19 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
                 "crystalkv_validate_static: the handle has " + std::to_string(total) + " pool slots, the built-in "
                 "scratch covers " + std::to_string(STATIC_SEEN_SLOTS) + "; use crystalkv_validate");
   if (c.device >= STATIC_MAX_DEVICES) return fail(h, CRYSTALKV_EINVAL, "crystalkv_validate_static: device ordinal above 63");
-  CK(h, cudaSetDevice(c.device));
-  if (!g_seen_addr[c.device]) {
+  ON_DEVICE(h);
+  int* seen = nullptr;
+  {
     // In host code the array's name is only a handle for the runtime; its device address has
     // to be asked for, once per device and with that device current.
-    int* addr = nullptr;
-    CK(h, cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_seen_static));
-    g_seen_addr[c.device] = addr;
+    std::lock_guard<std::mutex> lock(g_seen_mu);
+    if (!g_seen_addr[c.device]) {
+      int* addr = nullptr;
+      CK(h, cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_seen_static));
+      g_seen_addr[c.device] = addr;
+    }
+    seen = g_seen_addr[c.device];
   }
-  int* seen = g_seen_addr[c.device];
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   // the array keeps what the last call left: everything this call reads starts from zero
@@ -849,11 +905,13 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
 int crystalkv_join(crystalkv_t* h, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
   if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  ON_DEVICE(h);
   return join_side(h, static_cast<cudaStream_t>(stream));
 }
 
 int crystalkv_check(crystalkv_t* h, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   int w = 0;

@@ -22,6 +22,21 @@ def steps(n):
     return max(8, int(n * SCALE))
 
 
+def report(name, ls, note=""):
+    """One line per run: what was covered.  Printed, and appended to the file named by
+    CRYSTALKV_PARITY_REPORT when that is set."""
+    r = ls.rep
+    line = (f"{name}: sampled seqs {ls.seqs}, steps={r.steps} heads_compared={r.heads_compared} "
+            f"ties_logged={r.ties_logged} tie_explained={r.tie_explained} (each verified by a flipped replay; "
+            f"{r.replays} replays) unexplained={len(r.unexplained)} budgets_compared={r.budgets_compared} "
+            f"max_out_err={r.max_out_err:.3e}{note}")
+    print(line)
+    path = os.environ.get("CRYSTALKV_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+
+
 def test_cfg1_every_step_of_the_full_run():
     """Config 1 exactly: 256-token prompt, 2048 think steps, budget 512, state compared every step."""
     wl = WORKLOADS["cfg1_gqa4_b512"]
@@ -31,9 +46,7 @@ def test_cfg1_every_step_of_the_full_run():
     for _ in range(wl.think_steps):
         ls.step()
     ls.gpu.check()
-    r = ls.rep
-    print(f"cfg1: steps={r.steps} heads_compared={r.heads_compared} ties_logged={r.ties_logged} "
-          f"tie_explained={r.tie_explained} unexplained={len(r.unexplained)} max_out_err={r.max_out_err:.3e}")
+    report("cfg1_gqa4_b512", ls, " (state compared after every step)")
     ls.assert_clean()
     for h in range(2):
         assert len(ls.gpu.get_retained(0, 0, h)) == 512
@@ -168,24 +181,25 @@ def _run_sampled(name, sample, n_steps, cmp_every, answer=0, max_answer=0):
             ls.step(compare_state=False)
         ls.compare()
     ls.gpu.check()
-    r = ls.rep
-    print(f"{name}: sampled seqs {sample}, steps={r.steps} heads_compared={r.heads_compared} "
-          f"ties_logged={r.ties_logged} tie_explained={r.tie_explained} unexplained={len(r.unexplained)} "
-          f"budgets_compared={r.budgets_compared} max_out_err={r.max_out_err:.3e}")
+    report(name, ls, f" (state compared every {cmp_every} steps and around every reallocation)")
     ls.assert_clean()
     return ls
 
 
 def test_cfg2_qwen7b_shape_sampled():
-    """7B shape (28 layers, 28q/4kv, batch 8, budget 1024): past the point where heads fill."""
-    ls = _run_sampled("cfg2_qwen7b", [0, 7], steps(560), 40)
+    """7B shape (28 layers, 28q/4kv, batch 8, budget 1024): 512 steps to fill every head, then
+    more than 500 steps in which Algorithm 1 step 4 runs on every head."""
+    ls = _run_sampled("cfg2_qwen7b", [7], steps(1056), 32)
     assert len(ls.gpu.get_retained(27, 7, 3)) == 1024
     ls.close()
 
 
 def test_cfg3_llama8b_shape_sampled():
-    """8B shape (32 layers, 32q/8kv, batch 16, B_total = 2048 x heads), reallocation every 128."""
-    ls = _run_sampled("cfg3_llama8b", [15], steps(384), 32)
+    """8B shape (32 layers, 32q/8kv, batch 16, B_total = 2048 x heads), reallocation every 128:
+    past the point where the cache of a sequence is full (1536 steps after a 512-token prompt), so
+    that the last reallocations move slots between full heads and step 4 runs everywhere."""
+    ls = _run_sampled("cfg3_llama8b", [15], steps(1728), 32)
+    assert ls.rep.budgets_compared >= (13 if SCALE >= 1 else 0)
     b = ls.gpu.get_budgets()
     assert (b.reshape(16, -1).sum(axis=1) == 2048 * 32 * 8).all()
     ls.close()
@@ -194,7 +208,8 @@ def test_cfg3_llama8b_shape_sampled():
 def test_cfg4_qwen14b_shape_sampled():
     """14B shape (48 layers, 40q/8kv, batch 32, B_total = 1024 x heads), reallocation every 128,
     then answer steps: the configuration the bench times."""
-    ls = _run_sampled("cfg4_qwen14b", [31], steps(384), 32, answer=4, max_answer=8)
+    ls = _run_sampled("cfg4_qwen14b", [31], steps(1024), 32, answer=4, max_answer=8)
+    assert ls.rep.budgets_compared >= (8 if SCALE >= 1 else 0)
     b = ls.gpu.get_budgets()
     assert (b.reshape(32, -1).sum(axis=1) == 1024 * 48 * 8).all() and (b != 1024).any()
     ls.close()
@@ -342,6 +357,29 @@ def test_host_buffer_steps_match_device_steps():
         kv.check()
         kv.validate()
         kv.close()
+
+
+def test_a_smaller_handle_created_later_leaves_a_larger_one_working():
+    """Function attributes (the attention kernel's shared-memory limit) are per function, not per
+    handle: a handle with few heads created after one with many must not lower them."""
+    from paper_2601_16986_b200 import Config, CrystalKV
+    wl = Workload(name="many", seed=71, n_layers=1, n_q_heads=16, n_kv_heads=8, batch=200, prompt=20,
+                  think_steps=12, budget_per_head=24)
+    ls = LockStep(wl, [0, 199])
+    ls.prefill()
+    for _ in range(4):
+        ls.step()
+    small = CrystalKV(Config(n_layers=1, n_q_heads=2, n_kv_heads=1, batch=1, budget_per_head=8, max_context=64))
+    z = torch.zeros(1, 6, 1, 128, dtype=torch.bfloat16, device="cuda")
+    small.prefill(0, z, z, torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda"))
+    small.decode_step(0, torch.zeros(1, 2, 128, dtype=torch.bfloat16, device="cuda"), z[:, 0], z[:, 0])
+    small.check()
+    for _ in range(8):
+        ls.step()                       # the larger handle still launches
+    ls.gpu.check()
+    ls.assert_clean()
+    small.close()
+    ls.close()
 
 
 # ------------------------------------------------------------------ error paths on a live handle

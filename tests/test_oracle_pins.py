@@ -696,3 +696,54 @@ def test_export_import_round_trip():
             for h in range(2):
                 assert (a.export_state(l, s, h) == b.export_state(l, s, h)).all()
     a.close(); b.close()
+
+
+def test_replay_of_one_head_follows_the_run_and_a_flip_moves_one_entry():
+    """The harness's replay hook: with no flip it reproduces the oracle's own next states from an
+    exported state; a flip changes exactly the entry next to the hit boundary (the best-scored
+    miss becomes a hit, the worst-scored hit a miss, or both)."""
+    G = 2
+    w = tiny(n_q_heads=2 * G, n_kv_heads=2, prompt=10, think_steps=30, budget_per_head=64, seed=13, top_p=0.7)
+    o = make_oracle(w)
+    k, v = w.prompt_kv(0)
+    o.prefill(0, k, v, w.queries(0, [w.prompt - 1])[:, 0])
+    t0 = w.prompt + 9
+    for t in range(w.prompt, t0 + 1):
+        o.decode_step(0, *w.step_inputs(0, t))
+    h = 1
+    rec0 = o.export_state(0, 0, h)
+    pos0 = rec0[:, 0].tolist()
+    k0, v0 = w.keys(0, pos0)[0, :, h], w.values(0, pos0)[0, :, h]
+    steps = list(range(t0 + 1, t0 + 6))
+    q = w.queries(0, steps)[0, :, h * G:(h + 1) * G].contiguous()
+    kn, vn = w.keys(0, steps)[0, :, h].contiguous(), w.values(0, steps)[0, :, h].contiguous()
+    for t in steps:
+        o.decode_step(0, *w.step_inputs(0, t))
+    plain = o.replay_unit(rec0, k0, v0, 64, steps[0], q, kn, vn, np.zeros(5, dtype=np.int32))
+    assert (plain == o.export_state(0, 0, h)).all()
+    # one step, each flip: who changes
+    one = o.replay_unit(rec0, k0, v0, 64, steps[0], q[:1], kn[:1], vn[:1], np.array([0], dtype=np.int32))
+    posn = one[:, 0].tolist()
+    K = np.stack([f64(x) for x in w.keys(0, posn)[0, :, h]])
+    prob, _ = naive_attention(f64(q[0]), K, K, 1.0 / np.sqrt(w.head_dim))
+    pbar = prob.mean(axis=0)
+    hit = (one[:, 2] == steps[0]) & ~((one[:, 0] == steps[0]) & (one[:, 1] == 0))   # the arriving entry has tau = t either way
+    assert hit.any() and (~hit).any()
+    best_miss = int(np.flatnonzero(~hit)[np.argmax(pbar[~hit])])
+    worst_hit = int(np.flatnonzero(hit)[np.argmin(pbar[hit])])
+    for flip, changed in ((1, {best_miss}), (2, {worst_hit}), (3, {best_miss, worst_hit})):
+        alt = o.replay_unit(rec0, k0, v0, 64, steps[0], q[:1], kn[:1], vn[:1], np.array([flip], dtype=np.int32))
+        assert alt.shape == one.shape
+        assert set(np.flatnonzero((alt != one).any(axis=1)).tolist()) == changed
+        for i in changed:
+            assert alt[i, 1] != one[i, 1]        # its CRF took, or lost, the hit's "+ 1"
+    # the prefill's scoring pass as a replay: prompt entries with CRF 0 and tau = P - 1, nothing arrives
+    o2 = make_oracle(w)
+    o2.prefill(0, k, v, w.queries(0, [w.prompt - 1])[:, 0])
+    P = w.prompt
+    recp = np.stack([np.arange(P), np.zeros(P, dtype=np.int64), np.full(P, P - 1)], axis=1).astype(np.int32)
+    qp = w.queries(0, [P - 1])[0, :, h * G:(h + 1) * G].contiguous()
+    got = o2.replay_unit(recp, k[0, :, h], v[0, :, h], 64, P - 1, qp, k[0, P - 1:P, h].contiguous(),
+                         v[0, P - 1:P, h].contiguous(), np.zeros(1, dtype=np.int32), append_first=False)
+    assert (got == o2.export_state(0, 0, h)).all()
+    o.close(); o2.close()

@@ -1,8 +1,8 @@
 """crystalkv_validate_static: the slot-ownership check for callers that cannot allocate.
 
 Some users of this library run where a cudaMalloc is not an option: an inference server
-whose memory pool has already claimed the whole GPU, code that runs while a stream is being
-captured into a graph, a loop that cannot afford the device-wide stall of an allocation.
+whose memory pool has already claimed the whole GPU, or a loop that cannot afford the
+device-wide stall of an allocation.
 For them the library offers crystalkv_validate_static, which keeps its per-slot counters in
 an array built into the library instead of a temporary.  These tests call it through the C
 ABI and hold it against crystalkv_validate, the allocating entry point: same verdict on the
