@@ -593,6 +593,7 @@ def main():
         barrier()
         c0 = kv.get_counters()
         del rb_events[:]
+        launches["n"] = 0
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(stream)
         for s in range(s0, s1):

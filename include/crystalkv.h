@@ -145,8 +145,9 @@ int crystalkv_decode_step_host(crystalkv_t* h, int layer, const void* q_host,
  */
 int crystalkv_join(crystalkv_t* h, void* stream);
 
-/* Think stage: Algorithm 1 runs.  Answer stage: the think cache is frozen, new tokens
- * are appended beyond the budget and attended, nothing is tracked or evicted. */
+/* Section 4 splits a generation into the think stage, whose cache is compressed, and the
+ * answer stage.  Think stage: Algorithm 1 runs.  Answer stage: the think cache is frozen, new
+ * tokens are appended beyond the budget and attended, nothing is tracked or evicted. */
 int crystalkv_set_stage(crystalkv_t* h, int stage);
 
 /*
@@ -159,31 +160,50 @@ int crystalkv_set_stage(crystalkv_t* h, int stage);
 int crystalkv_rebudget(crystalkv_t* h, void* stream);
 
 /*
- * Token positions retained by (layer, seq, kv_head), ascending, into host memory.
- * Synchronises `stream`.  *n_out receives the count; ESTATE if cap is too small.
+ * Algorithm 1's output `Retain` as token positions: those kept by (layer, seq, kv_head),
+ * ascending, into host memory.  Synchronises `stream`.  *n_out receives the count; ESTATE if
+ * cap is too small.
  */
 int crystalkv_get_retained(crystalkv_t* h, int layer, int seq, int kv_head,
                            int32_t* pos_out_host, int32_t cap, int32_t* n_out, void* stream);
 
-/* Current budgets, host int32 [batch][L][H].  Synchronises `stream`. */
+/* Algorithm 2's output B': the current budgets, host int32 [batch][L][H].  Synchronises `stream`. */
 int crystalkv_get_budgets(crystalkv_t* h, int32_t* out_host, void* stream);
 
 /*
- * Per-entry state of one head, sorted by position: records of three int32
- * {position, CRF as fp32 bits, tau}.  host_buf holds cap records; *n receives the
- * count.  Synchronises `stream`.
+ * The state Algorithm 1 keeps per entry of one head (its inputs CRF and tau, next to the
+ * entry's token position), sorted by position: records of three int32 {position, CRF as fp32
+ * bits, tau}.  host_buf holds cap records; *n receives the count.  Synchronises `stream`.
  */
 int crystalkv_export_state(crystalkv_t* h, int layer, int seq, int kv_head, int32_t* host_buf,
                            int32_t cap, int32_t* n, void* stream);
 
 /*
- * Overwrites CRF and tau of the listed positions (records as in export).  Every
- * position must be present in the head's cache (else ESTATE, nothing changed).
+ * The other two inputs of Algorithm 1, K and V, of one head: its entries' rows in the order
+ * of crystalkv_export_state's records, host bf16 [n][128] each (cap rows of room).  *n
+ * receives the count.  Synchronises `stream`.
+ */
+int crystalkv_export_kv(crystalkv_t* h, int layer, int seq, int kv_head, void* k_rows_host,
+                        void* v_rows_host, int32_t cap, int32_t* n, void* stream);
+
+/*
+ * The inverse of the two exports: replaces the content of one head by n entries given as
+ * records {position, CRF bits, tau} (any order) with their K and V rows, host bf16 [n][128]
+ * each, and sets the head's budget (Algorithm 1's input B; 0 keeps the current one) and the
+ * layer's time t (the time of its last completed step, Algorithm 1's input t).  The head returns
+ * the pool pages it no longer needs and takes those it lacks.  A layer that was never
+ * prefilled becomes usable once every one of its heads has been imported with the same t: a
+ * handle can be rebuilt from the exports of another (with crystalkv_set_stage for the stage).
+ * Synchronises `stream`.  Errors: EINVAL (n outside [1, list capacity), budget outside
+ * [0, max_budget], a position or tau after t), ESTATE (the layer is at another time), ECHECK
+ * later from crystalkv_check if the sequence's pool had no pages left.
  */
 int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head,
-                           const int32_t* host_buf, int32_t n, void* stream);
+                           const int32_t* host_buf, int32_t n, const void* k_rows_host,
+                           const void* v_rows_host, int32_t budget, int32_t t, void* stream);
 
-/* Sets one head's budget directly (tests and checkpoint restore). */
+/* Sets one head's budget (Algorithm 1's input B) directly; a head holding more evicts down to
+ * it at once, as after a reallocation. */
 int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_t budget,
                          void* stream);
 
@@ -202,9 +222,10 @@ int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t*
 int crystalkv_check(crystalkv_t* h, void* stream);
 
 /*
- * Debug check of slot ownership (the in-place slot reuse of Algorithm 1 step 4 and the
- * slot hand-over of the reallocation): every pool slot of every sequence must be held
- * exactly once, by the sequence's free list or by one head (entries plus one spare).
+ * Debug check of page ownership (the in-place reuse of Algorithm 1 step 4 and the hand-over
+ * of pool pages between heads by the reallocation): every pool page (16 entries) of every
+ * sequence must be held exactly once, by the sequence's free list or by one head, and every
+ * head must hold the pages that back its entries and the place of its next arrival.
  * Allocates a temporary, synchronises `stream`; not for the hot path.  ECHECK on failure,
  * ESTATE before every layer is prefilled.
  */
@@ -218,27 +239,28 @@ int crystalkv_validate(crystalkv_t* h, void* stream);
  * where a framework has already claimed all device memory for its own pool (cudaMalloc then
  * fails although the framework has room), or in a serving loop that may not take the
  * device-wide synchronisation a cudaMalloc / cudaFree pair implies.  This entry point does the
- * same check with its per-slot counters in an array that is built into the library: it calls
+ * same check with its per-page counters in an array that is built into the library: it calls
  * no cudaMalloc, cudaFree or other allocating routine.  Like crystalkv_validate it copies its
  * verdict to the host and synchronises `stream`, so it is not a call for a stream that is
  * being captured.
  *
- *   counts_out_host  host int32[2] or NULL: [0] slot ids out of range, [1] slots not owned
- *                    exactly once (both 0 on a sound handle)
+ *   counts_out_host  host int32[2] or NULL: [0] page ids or counts out of range, [1] pages not
+ *                    owned exactly once (both 0 on a sound handle)
  *
  * Limits and rules
- *   - The array covers handles of at most 2^21 = 2 097 152 pool slots in total (1 GiB of K/V
- *     rows): batch * L * H * (budget_per_head + evict_every + max_answer_tokens) slots in evict
- *     mode, batch * L * H * (max_context + 1) in FullKV mode.  A larger handle is refused with
- *     EINVAL and a message that says so; use crystalkv_validate there.
- *   - Every GPU on which the library is loaded holds the array (8 MiB) until the process ends.
+ *   - The array covers handles of at most 2^17 = 131 072 pool pages in total (1 GiB of K/V
+ *     rows).  A handle has batch * (ceil(L * H * E / 16) + L * H) pages, with E = budget_per_head
+ *     + evict_every + max_answer_tokens + 1 entries per head in evict mode and max_context + 1
+ *     in FullKV mode.  A larger handle is refused with EINVAL and a message that says so; use
+ *     crystalkv_validate there.
+ *   - Every GPU on which the library is loaded holds the array (512 KiB) until the process ends.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress,
  *     with that device made current).  Make that first call before any stream capture begins.
  *   - All calls on one GPU, from any handle, share the array, and it keeps the previous
  *     call's contents; each call clears the part it uses on `stream` first.  Two calls whose
  *     work overlaps on the GPU (different streams, no ordering between them) race: order them.
  *   - Like crystalkv_validate it synchronises `stream` and is not for the hot path.
- * Errors: EINVAL (NULL handle, too many slots, device ordinal above 63), ESTATE before every
+ * Errors: EINVAL (NULL handle, too many pages, device ordinal above 63), ESTATE before every
  * layer is prefilled, ECUDA, ECHECK when ownership is broken.
  */
 int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* stream);

@@ -90,7 +90,8 @@ def load_library():
     lib.crystalkv_get_retained.argtypes = [vp, i32, i32, i32, vp, C.c_int32, p32, vp]
     lib.crystalkv_get_budgets.argtypes = [vp, vp, vp]
     lib.crystalkv_export_state.argtypes = [vp, i32, i32, i32, vp, C.c_int32, p32, vp]
-    lib.crystalkv_import_state.argtypes = [vp, i32, i32, i32, vp, C.c_int32, vp]
+    lib.crystalkv_export_kv.argtypes = [vp, i32, i32, i32, vp, vp, C.c_int32, p32, vp]
+    lib.crystalkv_import_state.argtypes = [vp, i32, i32, i32, vp, C.c_int32, vp, vp, C.c_int32, C.c_int32, vp]
     lib.crystalkv_set_budget.argtypes = [vp, i32, i32, i32, C.c_int32, vp]
     lib.crystalkv_time.argtypes = [vp, i32]
     lib.crystalkv_get_counters.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
@@ -219,10 +220,24 @@ class CrystalKV:
                                                  self._cap, C.byref(n), _stream()))
         return buf[:n.value].copy()
 
-    def import_state(self, layer, seq, kv_head, rec: np.ndarray):
+    def export_kv(self, layer, seq, kv_head):
+        """K and V rows of one head in the order of export_state's records: two host bf16 tensors [n, 128]."""
+        k = torch.empty(self._cap, self.cfg.head_dim, dtype=torch.bfloat16)
+        v = torch.empty(self._cap, self.cfg.head_dim, dtype=torch.bfloat16)
+        n = C.c_int32(0)
+        self._ck(self.lib.crystalkv_export_kv(self._h, layer, seq, kv_head, C.c_void_p(k.data_ptr()),
+                                              C.c_void_p(v.data_ptr()), self._cap, C.byref(n), _stream()))
+        return k[:n.value].clone(), v[:n.value].clone()
+
+    def import_state(self, layer, seq, kv_head, rec: np.ndarray, k: torch.Tensor, v: torch.Tensor, budget: int, t: int):
+        """Rebuilds one head from records [n, 3] and host bf16 rows k, v [n, 128]; budget 0 keeps the current one."""
         rec = np.ascontiguousarray(rec, dtype=np.int32)
-        self._ck(self.lib.crystalkv_import_state(self._h, layer, seq, kv_head, rec.ctypes.data_as(C.c_void_p),
-                                                 len(rec), _stream()))
+        for x in (k, v):
+            if x.is_cuda or x.dtype != torch.bfloat16 or not x.is_contiguous() or tuple(x.shape) != (len(rec), self.cfg.head_dim):
+                raise ValueError("expected contiguous host bf16 rows [n, head_dim]")
+        self._ck(self.lib.crystalkv_import_state(self._h, layer, seq, kv_head, rec.ctypes.data_as(C.c_void_p), len(rec),
+                                                 C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()), int(budget), int(t),
+                                                 _stream()))
 
     def set_budget(self, layer, seq, kv_head, budget):
         self._ck(self.lib.crystalkv_set_budget(self._h, layer, seq, kv_head, int(budget), _stream()))
@@ -243,7 +258,7 @@ class CrystalKV:
 
     def validate_static(self) -> np.ndarray:
         """The same check without any device allocation (scratch built into the library; at
-        most 2**21 pool slots).  Returns int32[2]: ids out of range, slots not owned once."""
+        most 2**17 pool pages).  Returns int32[2]: ids out of range, slots not owned once."""
         counts = np.full(2, -1, dtype=np.int32)
         self._ck(self.lib.crystalkv_validate_static(self._h, counts.ctypes.data_as(C.c_void_p), _stream()))
         return counts

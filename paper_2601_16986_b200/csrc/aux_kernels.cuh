@@ -7,53 +7,58 @@
 namespace ckv {
 
 // ---------------------------------------------------------------------------------------
-// Prompt insertion for one layer: one CTA per (sequence, kv head).  Takes P + 1 slots from the
-// sequence's free list (P entries and the spare), copies the K/V rows into them and sets
-// pos = i, CRF = 0 and tau = P - 1 (the time of the scoring pass that follows) or, when the
-// prompt's last tokens are replayed one by one, tau = i (the token's own arrival time).
+// Prompt insertion for one layer: one CTA per (sequence, kv head).  Takes the pages that back
+// list positions 0 .. P (the P entries and the place of the next arrival) from the sequence's
+// free list, writes the K/V rows into them in the page layout and sets pos = i, CRF = 0 and
+// tau = P - 1 (the time of the scoring pass that follows) or, when the prompt's last tokens
+// are replayed one by one, tau = i (the token's own arrival time).
 //   k, v: [batch][P][H][128] bf16
-__global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int* n_out, int layer,
-                                                            const __nv_bfloat16* k,
+__global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int layer, const __nv_bfloat16* k,
                                                             const __nv_bfloat16* v, int P, int tau_is_pos) {
   __shared__ int s_top;
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
   const int uid = (seq * st.L + layer) * st.H + head;
   const size_t mb = (size_t)uid * st.cap;
   const int tid = threadIdx.x;
+  const int need = P / GRP + 1;
   if (tid == 0) {
-    int top = atomicSub(&st.free_top[seq], P + 1);
-    if (top < P + 1) {
-      atomicAdd(&st.free_top[seq], P + 1);
-      atomicOr(st.errword, ERR_FREE_UNDERFLOW);
-      top = -1;
+    int top = -1;
+    if (P + 1 > st.cap) {
+      atomicOr(st.errword, ERR_CAPACITY);
+    } else {
+      top = atomicSub(&st.free_top[seq], need);
+      if (top < need) {
+        atomicAdd(&st.free_top[seq], need);
+        atomicOr(st.errword, ERR_FREE_UNDERFLOW);
+        top = -1;
+      }
     }
     s_top = top;
   }
   __syncthreads();
   const int top = s_top;
   if (top < 0) {
-    if (tid == 0) n_out[uid] = 0;
+    if (tid == 0) { st.n_cur[uid] = 0; st.hole[uid] = 0; }
     return;
   }
-  if (tid == 0) st.own[uid] = P + 1;
-  const int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
-  for (int i = tid; i <= P; i += NT) {
-    st.list_slot[mb + i] = stack[top - 1 - i];
-    if (i < P) {
-      st.meta_pos[mb + i] = i;
-      st.meta_tau[mb + i] = tau_is_pos ? i : P - 1;
-      st.meta_crf[mb + i] = 0.0f;
-    }
+  const int* stack = st.free_stack + (size_t)seq * st.pages_per_seq;
+  int* pt = st.ptab + (size_t)uid * st.capg;
+  for (int j = tid; j < need; j += NT) pt[j] = stack[top - 1 - j];
+  for (int i = tid; i < P; i += NT) {
+    st.meta_pos[mb + i] = i;
+    st.meta_tau[mb + i] = tau_is_pos ? i : P - 1;
+    st.meta_crf[mb + i] = 0.0f;
   }
-  unsigned char* poolseq = st.pool + (size_t)seq * st.slots_per_seq * SLOT_BYTES;
-  const int piece = tid & 31;
+  unsigned char* poolseq = st.pool + (size_t)seq * st.pages_per_seq * PAGE_BYTES;
+  const int c = tid & 31;   // chunk of the entry's 512 bytes: K row, then V row
   for (int i = tid >> 5; i < P; i += NW) {
-    const int slot = stack[top - 1 - i];
+    const int page = stack[top - 1 - (i >> 4)];
     const size_t off = (((size_t)seq * P + i) * st.H + head) * HD * 2;
-    const unsigned char* src = reinterpret_cast<const unsigned char*>(piece < 16 ? k : v) + off + (piece & 15) * 16;
-    *reinterpret_cast<uint4*>(poolseq + (size_t)slot * SLOT_BYTES + piece * 16) = *reinterpret_cast<const uint4*>(src);
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(c < 16 ? k : v) + off + (c & 15) * 16;
+    *reinterpret_cast<uint4*>(poolseq + (size_t)page * PAGE_BYTES + chunk_offset(i & (GRP - 1), c)) =
+        *reinterpret_cast<const uint4*>(src);
   }
-  if (tid == 0) n_out[uid] = P;
+  if (tid == 0) { st.n_cur[uid] = P; st.hole[uid] = P; st.npages[uid] = need; }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -79,14 +84,14 @@ __global__ void __launch_bounds__(NT) stage_in_kernel(uint4* __restrict__ dq, ui
 // ---------------------------------------------------------------------------------------
 // Algorithm 2 input: per head, the sum of CRF decayed to t_last over the retained entries,
 // each term truncated to 2^-32 fixed point so the sum does not depend on the order.
-__global__ void __launch_bounds__(NT) crf_sum_kernel(State st, const int* n_cur, int t_last,
-                                                     long long* Asum) {
+__global__ void __launch_bounds__(NT) crf_sum_kernel(State st, int t_last, long long* Asum) {
   __shared__ long long s_red[NW];
   const int uid = blockIdx.x;
   const size_t mb = (size_t)uid * st.cap;
-  const int n = n_cur[uid];
+  const int n = st.n_cur[uid], hole = st.hole[uid];
   long long acc = 0;
-  for (int i = threadIdx.x; i < n; i += NT) {
+  for (int x = threadIdx.x; x < n; x += NT) {
+    const int i = live_pos(x, hole);
     const float d = __fmul_rn(st.tab[t_last - st.meta_tau[mb + i]], st.meta_crf[mb + i]);
     acc += (long long)((double)d * 4294967296.0);
   }
@@ -240,43 +245,59 @@ __global__ void __launch_bounds__(NT) alg2_kernel(const long long* Asum, int* bu
 }
 
 // ---------------------------------------------------------------------------------------
+// Makes a head's list dense: the last entry moves into the hole an evicted entry left (one row and
+// its metadata).  Needed before anything that works on a dense list outside a decode step.
+__device__ __forceinline__ void close_hole(const State& st, int uid, int seq) {
+  const int n = st.n_cur[uid], hole = st.hole[uid];
+  __syncthreads();
+  if (hole < n) {
+    if (threadIdx.x < 32) move_entry(st, uid, seq, (size_t)uid * st.cap, hole, n, threadIdx.x);
+    __syncthreads();
+    if (threadIdx.x == 0) st.hole[uid] = n;
+  }
+  __syncthreads();
+}
+
 // Shrink pass for the heads of one layer (one CTA per head): a head holding more entries than
-// its budget drops its lowest (decayed CRF, tau, pos) entries; their slots, beyond one spare,
-// go back to the sequence's free list, from which heads that grew refill step by step.
-__global__ void __launch_bounds__(NT) shrink_kernel(State st, int* n_cur, int layer, int t_last,
-                                                    int* tmp, int tmp_stride) {
+// its budget drops its lowest (decayed CRF, tau, pos) entries; the pages that become empty go
+// back to the sequence's free list, from which heads that grew refill step by step.
+__global__ void __launch_bounds__(NT) shrink_kernel(State st, int layer, int t_last, int* tmp, int tmp_stride) {
   __shared__ int sh[300];
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
   const int uid = (seq * st.L + layer) * st.H + head;
-  const int n = n_cur[uid], B = st.budget[uid];
+  const int n = st.n_cur[uid], B = st.budget[uid];
   if (n <= B || n < 2) return;
-  evict_many(st, n_cur, uid, seq, n, min(n - B, n - 1), t_last, true, sh, tmp + (size_t)u * tmp_stride);
+  close_hole(st, uid, seq);
+  evict_many(st, uid, seq, n, min(n - B, n - 1), t_last, true, sh, tmp + (size_t)u * tmp_stride);
 }
 
 // ---------------------------------------------------------------------------------------
-// Consistency check of slot ownership: every pool slot of a sequence must be owned exactly
-// once, either by the free list or by one head (its n entries and its spares).
+// Consistency check of page ownership: every pool page of a sequence must be owned exactly
+// once, either by the free list or by one head, and every head must own the pages that back its
+// entries and its hole.
 __global__ void mark_free_kernel(State st, int* seen) {
   const int seq = blockIdx.y;
   const int top = st.free_top[seq];
-  const int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
+  const int* stack = st.free_stack + (size_t)seq * st.pages_per_seq;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < top; i += (long long)gridDim.x * blockDim.x) {
     const int s = stack[i];
-    if (s < 0 || s >= st.slots_per_seq) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);
-    else atomicAdd(&seen[(size_t)seq * st.slots_per_seq + s], 1);
+    if (s < 0 || s >= st.pages_per_seq) atomicAdd(&seen[(size_t)st.batch * st.pages_per_seq], 1);
+    else atomicAdd(&seen[(size_t)seq * st.pages_per_seq + s], 1);
   }
 }
 
-__global__ void mark_owned_kernel(State st, const int* n_cur, int layer, int* seen) {
+__global__ void mark_owned_kernel(State st, int layer, int* seen) {
   const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
   const int uid = (seq * st.L + layer) * st.H + head;
-  const size_t mb = (size_t)uid * st.cap;
-  const int own = st.own[uid];
-  if (threadIdx.x == 0 && own < n_cur[uid] + 1) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);   // no spare
-  for (int i = threadIdx.x; i < own; i += blockDim.x) {   // the entries, then the spares
-    const int s = st.list_slot[mb + i];
-    if (s < 0 || s >= st.slots_per_seq) atomicAdd(&seen[(size_t)st.batch * st.slots_per_seq], 1);
-    else atomicAdd(&seen[(size_t)seq * st.slots_per_seq + s], 1);
+  const int own = st.npages[uid];
+  if (threadIdx.x == 0) {
+    const int n = st.n_cur[uid], hole = st.hole[uid];
+    if (own * GRP <= n || own > st.capg || hole < 0 || hole > n) atomicAdd(&seen[(size_t)st.batch * st.pages_per_seq], 1);
+  }
+  for (int j = threadIdx.x; j < min(own, st.capg); j += blockDim.x) {
+    const int s = st.ptab[(size_t)uid * st.capg + j];
+    if (s < 0 || s >= st.pages_per_seq) atomicAdd(&seen[(size_t)st.batch * st.pages_per_seq], 1);
+    else atomicAdd(&seen[(size_t)seq * st.pages_per_seq + s], 1);
   }
 }
 
@@ -286,6 +307,75 @@ __global__ void count_bad_kernel(const int* seen, long long total, int* bad) {
     loc += (seen[i] != 1);
   loc = warp_sum_i(loc);
   if ((threadIdx.x & 31) == 0 && loc) atomicAdd(bad, loc);
+}
+
+// ---------------------------------------------------------------------------------------
+// State of one head for the host, entry by entry in list order (the hole skipped): records
+// {position, CRF bits, tau} and, when asked for, the K and V rows in plain row layout.
+__global__ void __launch_bounds__(NT) export_unit_kernel(State st, int uid, int seq, int* rec, unsigned char* krows,
+                                                         unsigned char* vrows, int* n_out) {
+  const int n = st.n_cur[uid], hole = st.hole[uid];
+  const size_t mb = (size_t)uid * st.cap;
+  if (threadIdx.x == 0) *n_out = n;
+  for (int x = threadIdx.x; x < n; x += NT) {
+    const int i = live_pos(x, hole);
+    rec[3 * x] = st.meta_pos[mb + i];
+    rec[3 * x + 1] = __float_as_int(st.meta_crf[mb + i]);
+    rec[3 * x + 2] = st.meta_tau[mb + i];
+  }
+  if (!krows) return;
+  const int c = threadIdx.x & 31;
+  for (int x = threadIdx.x >> 5; x < n; x += NW) {
+    const uint4 v = *reinterpret_cast<const uint4*>(entry_chunk(st, uid, seq, live_pos(x, hole), c));
+    *reinterpret_cast<uint4*>((c < 16 ? krows : vrows) + (size_t)x * ROW_BYTES + (c & 15) * 16) = v;
+  }
+}
+
+// The inverse: replaces the head's content by n entries given as records and rows (in any
+// order; they become list positions 0 .. n-1), returns the pages it no longer needs and takes
+// those it lacks.  One CTA; no other kernel that takes or returns pages runs beside it.
+__global__ void __launch_bounds__(NT) import_unit_kernel(State st, int uid, int seq, const int* rec, const unsigned char* krows,
+                                                         const unsigned char* vrows, int n, int budget) {
+  __shared__ int s_base;
+  const int tid = threadIdx.x;
+  const int need = n / GRP + 1;
+  int have = st.npages[uid];
+  if (n + 1 > st.cap) {
+    if (tid == 0) atomicOr(st.errword, ERR_CAPACITY);
+    return;
+  }
+  if (have > need) {
+    release_pages(st, uid, seq, n, &s_base);
+  } else if (have < need) {
+    if (tid == 0) {
+      int top = atomicSub(&st.free_top[seq], need - have);
+      if (top < need - have) {
+        atomicAdd(&st.free_top[seq], need - have);
+        atomicOr(st.errword, ERR_FREE_UNDERFLOW);
+        top = -1;
+      }
+      s_base = top;
+    }
+    __syncthreads();
+    if (s_base < 0) return;
+    const int* stack = st.free_stack + (size_t)seq * st.pages_per_seq;
+    for (int j = tid; j < need - have; j += NT) st.ptab[(size_t)uid * st.capg + have + j] = stack[s_base - 1 - j];
+    __syncthreads();
+    if (tid == 0) st.npages[uid] = need;
+  }
+  __syncthreads();
+  const size_t mb = (size_t)uid * st.cap;
+  for (int i = tid; i < n; i += NT) {
+    st.meta_pos[mb + i] = rec[3 * i];
+    st.meta_crf[mb + i] = __int_as_float(rec[3 * i + 1]);
+    st.meta_tau[mb + i] = rec[3 * i + 2];
+  }
+  const int c = tid & 31;
+  for (int i = tid >> 5; i < n; i += NW) {
+    const uint4 v = *reinterpret_cast<const uint4*>((c < 16 ? krows : vrows) + (size_t)i * ROW_BYTES + (c & 15) * 16);
+    *reinterpret_cast<uint4*>(entry_chunk(st, uid, seq, i, c)) = v;
+  }
+  if (tid == 0) { st.n_cur[uid] = n; st.hole[uid] = n; st.budget[uid] = budget; }
 }
 
 }  // namespace ckv

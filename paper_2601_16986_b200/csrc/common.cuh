@@ -8,50 +8,70 @@ namespace ckv {
 
 constexpr int HD = 128;             // head_dim
 constexpr int ROW_BYTES = 256;      // one K or V row, bf16
-constexpr int SLOT_BYTES = 512;     // pool slot = K row followed by V row
-constexpr int GRP = 16;             // keys per streamed group (one MMA tile of keys)
+constexpr int SLOT_BYTES = 512;     // one entry in the pool: K row followed by V row
+constexpr int GRP = 16;             // entries per page = keys per streamed group (one MMA tile of keys)
+constexpr int PAGE_BYTES = GRP * SLOT_BYTES;   // 8 KB: what one bulk copy brings into a ring stage
 constexpr int NW = 8;               // warps per CTA
 constexpr int NT = NW * 32;
-constexpr int STAGES = 3;           // ring depth per warp, in groups
-constexpr int STAGE_BYTES = GRP * (SLOT_BYTES + 16);   // 16 entries, each K row + V row + 16 B of padding
-constexpr int RING_BYTES = NW * STAGES * STAGE_BYTES;  // 198 KB
-constexpr int GMIN = 4;             // fewest groups a working warp takes
+constexpr int STAGES = 3;           // ring depth per warp, in pages
+constexpr int RING_BYTES = NW * STAGES * PAGE_BYTES;   // 192 KB
+constexpr int GMIN = 4;             // fewest groups a streaming warp is given
 constexpr int QH = 8;               // query heads of a group as padded for the MMA N dimension
-constexpr int MAX_UNITS_PER_CALL = 2048;   // bounded by the split tables in shared memory
-constexpr int NSETS = 16;           // logit scratch sets cycled by consecutive tracked launches
+constexpr int MAX_UNITS_PER_CALL = 2048;   // heads of one layer launch (bounded by the planner's shared memory)
+constexpr int NSETS = 16;           // logit scratch sets cycled by consecutive launches
+constexpr int FIFO = 8;             // pieces a warp may have fetched ahead of the one it computes (> STAGES)
 
 // error word bits raised by device-side consistency checks (never a trap)
-constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a slot and the sequence's free list was empty
+constexpr int ERR_FREE_UNDERFLOW = 1;   // a head needed a page and the sequence's free list was empty
 constexpr int ERR_OVER_EVICT = 2;       // a decode step found a head further over its budget than the eviction period allows
 constexpr int ERR_CAPACITY = 4;         // a head's list would outgrow its capacity
 constexpr int ERR_NUCLEUS = 8;          // the top-p threshold search did not find its boundary
 constexpr int ERR_COPY_TIMEOUT = 16;    // a bulk copy into shared memory did not complete within a second
+constexpr int ERR_PLAN = 32;            // the launch plan of a layer does not match the grid it is used with
+
+// Layout of a pool page: entry e (0..15) occupies bytes [512 e, 512 e + 512): its K row, then its
+// V row, as 32 chunks of 16 bytes; chunk c is stored at chunk index c ^ (e & 7).  A page copied
+// as it is into shared memory can then be read by ldmatrix (eight entries, one chunk column)
+// without bank conflicts, and one bulk copy brings a whole group of keys.
+__host__ __device__ __forceinline__ int chunk_offset(int e, int c) { return e * SLOT_BYTES + ((c ^ (e & 7)) << 4); }
 
 struct State {
-  // K/V pool: [batch][slots_per_seq][512 B]
+  // K/V pool: [batch][pages_per_seq][8192 B]
   unsigned char* pool;
-  long long slots_per_seq;
-  int* free_stack;   // [batch][slots_per_seq]
-  int* free_top;     // [batch] number of free slots
-  // per unit (uid = (seq*L + layer)*H + head), capacity `cap` list positions
-  int* list_slot;    // [units][cap] slot of the entry at a list position; position n holds the spare
+  long long pages_per_seq;
+  int* free_stack;   // [batch][pages_per_seq] free page ids of a sequence
+  int* free_top;     // [batch] number of free pages
+  // per unit (uid = (seq*L + layer)*H + head): `cap` list positions, page j backs positions 16 j .. 16 j + 15
+  int* ptab;         // [units][capg] page id per 16 list positions; the first npages are owned by the unit
   int* meta_pos;     // [units][cap] token position
   int* meta_tau;     // [units][cap] last hit time
   float* meta_crf;   // [units][cap] CRF at tau
-  int* nbuf[2];      // [2][units] entry counts, double buffered: a step reads one and writes the other
+  int* n_cur;        // [units] live entries
+  int* hole;         // [units] list position the next arriving entry is written to (<= n).  The live entries
+                     // are the positions 0 .. n without the hole (hole == n: positions 0 .. n-1).  An entry that
+                     // leaves in a decode step leaves its place to the next arrival: nothing is moved.
+  int* npages;       // [units] pages owned; 16 * npages > n always (the hole is backed)
   int* budget;       // [units] == [batch][L][H]
-  int* own;          // [units] list positions [0, own) hold slots that belong to the head: its entries, then
-                     // its spares (one in steady state; up to the eviction period with a buffered cadence)
   const float* tab;  // lambda^D, D in [0, max_context]
   int* errword;
   unsigned long long* counters;  // entries attended, hits, evictions
-  int batch, L, H, cap;
+  int batch, L, H, cap, capg;
+};
+
+// Launch plan of one layer, written by the kernel that last changed the layer's lengths and read
+// by the next attention launch: all groups of the layer's heads laid in a row and cut into
+// nearly equal runs, one run per streaming warp; a run is one piece per head it overlaps.
+struct Plan {
+  int4* desc;        // [pd_cap] pieces in row order: {head index u, first group, end group, (pieces of u << 16) | piece index}
+  int2* wrange;      // [warps] pieces [x, y) of the physical warp cta * NW + w
+  int* npc;          // [U] pieces per head
+  int* hdr;          // [4] pieces in total, groups in total, warps the plan was made for, append it was made for
 };
 
 // scratch of one launch pair (attention kernel, then LRFU kernel), assembled per launch: the
 // logits and (m, l) come from one of NSETS cycled sets, the partials and tickets from one of two
 struct Scratch {
-  float* logits;     // [U][cap_s][QH] scaled logits of the step, one 32-byte row per entry
+  float* logits;     // [U][cap_s][QH] scaled logits of the step, one 32-byte row per list position
   float* pbar;       // [U][cap_s] group-mean probabilities (reused as int scratch)
   float* partials;   // [U][pmax][16 + G*128] split-K partial: m[8], l[8], O[G][128]
   float* mfin;       // [U][2][QH] per query head: merged reference point (log2 domain), then normaliser
@@ -62,26 +82,27 @@ struct Scratch {
 struct DecodeParams {
   State st;
   Scratch sc;
+  Plan plan;                    // of this layer
   const __nv_bfloat16* q;       // [batch][Hq][128]
   const __nv_bfloat16* k_new;   // [batch][H][128]
   const __nv_bfloat16* v_new;
   __nv_bfloat16* out;           // [batch][Hq][128]
-  int* piece_ctr;    // counters by launch parity: [0..1] the attention warps take pieces, [2..3] its CTAs take chunks of pieces
-  int parity;
-  const int* n_in;   // entry counts before this step
-  int* n_out;        // entry counts after it
+  int* done_ctr;     // LRFU kernel: counts its finished CTAs; the last one writes the layer's next plan
   int layer;
   int G;          // query heads per kv head
   int t;          // time of this step
   int append;     // 1: decode (a new entry arrives); 0: scoring pass over the prompt
   int track;      // 1: Algorithm 1 runs (hits, CRF, eviction) in the LRFU kernel that follows
-  int release;    // 1: freed slots beyond one spare go back to the free list (no pops in this launch)
+  int release;    // 1: pages a head no longer needs go back to the free list (no pops in this launch)
   int early;      // 1: the lists and rows of this layer are final, so the attention kernel may read them
                   //    before the kernel ahead of it in the stream has completed
   int n_limit;    // > 0: only the first n_limit entries of every head take part (a prompt token's causal view)
   int hold;       // 1: Algorithm 1 stops after step 3; lengths and lists stay as they are
   int evict_every;   // m >= 1: step 4 waits until a head is m entries over its budget, then removes them all
   int literal;    // 1: Algorithm 1 is skipped for a head below its budget (its first line as printed)
+  int plan_append;   // what the plan the LRFU kernel leaves behind is for: 1 = a decode step, 0 = a scoring pass
+  int plan_warps;    // warps of the attention grid the plan is made for
+  int plan_grid;     // CTAs of that grid
   float scale;    // logit scale
   float scale_log2;
   float top_p;
@@ -89,14 +110,6 @@ struct DecodeParams {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -150,14 +163,19 @@ __device__ __forceinline__ int block_excl_scan(int v, int* red, int& total) {
   return base + inc - v;
 }
 
-// A head keeps its length and, unless it still owns a spare there, takes a fresh slot for list
-// position n (decode steps in which nothing left the head).  One thread calls it.
-__device__ __forceinline__ void keep_and_refill(const State& st, int* n_out, int uid, int seq, int n,
-                                                bool append) {
-  n_out[uid] = n;
-  if (!append) return;
-  if (st.own[uid] > n) return;   // one of the head's own spares is at list position n already
-  if (n + 1 > st.cap) {
+// Address of chunk c (16 bytes) of the entry at list position i of a head.
+__device__ __forceinline__ unsigned char* entry_chunk(const State& st, int uid, int seq, int i, int c) {
+  const int page = st.ptab[(size_t)uid * st.capg + (i >> 4)];
+  return st.pool + ((size_t)seq * st.pages_per_seq + page) * PAGE_BYTES + chunk_offset(i & (GRP - 1), c);
+}
+
+// Makes sure list position `need` of a head is backed by a page (a head that grew past its last
+// page takes one from its sequence's free list).  One thread calls it; launches in which heads
+// return pages never call it.
+__device__ __forceinline__ void back_position(const State& st, int uid, int seq, int need) {
+  const int have = st.npages[uid];
+  if (need < have * GRP) return;
+  if (need >= st.cap) {
     atomicOr(st.errword, ERR_CAPACITY);
     return;
   }
@@ -166,9 +184,19 @@ __device__ __forceinline__ void keep_and_refill(const State& st, int* n_out, int
     atomicAdd(&st.free_top[seq], 1);
     atomicOr(st.errword, ERR_FREE_UNDERFLOW);
   } else {
-    st.list_slot[(size_t)uid * st.cap + n] = st.free_stack[(size_t)seq * st.slots_per_seq + idx];
-    st.own[uid] = n + 1;
+    st.ptab[(size_t)uid * st.capg + have] = st.free_stack[(size_t)seq * st.pages_per_seq + idx];
+    st.npages[uid] = have + 1;
   }
 }
+
+// A head keeps all n entries of a step: the next arrival goes behind them.
+__device__ __forceinline__ void keep_all(const State& st, int uid, int seq, int n, bool will_append) {
+  st.n_cur[uid] = n;
+  st.hole[uid] = n;
+  if (will_append) back_position(st, uid, seq, n);
+}
+
+// List position of the i-th live entry of a head (i in [0, n)) given its hole.
+__device__ __forceinline__ int live_pos(int i, int hole) { return i + (i >= hole ? 1 : 0); }
 
 }  // namespace ckv

@@ -24,6 +24,7 @@
 #include "attn_kernel.cuh"
 #include "aux_kernels.cuh"
 #include "lrfu_kernel.cuh"
+#include "plan.cuh"
 
 using namespace ckv;
 
@@ -31,8 +32,11 @@ struct crystalkv {
   crystalkv_config_t cfg;
   int G = 0, U = 0, units = 0, cap = 0, num_sms = 0, grid = 0;
   size_t smem = 0;
-  long long slots_per_seq = 0;
+  long long pages_per_seq = 0;
   State st{};
+  std::vector<Plan> plans;         // per layer: the launch plan of its next attention kernel
+  Plan* d_plans = nullptr;
+  int* done_ctr = nullptr;
   // scratch: logits and merged (m, l) per cycled set (the LRFU kernel reads them while later
   // attention kernels run), partials and tickets alternate between two (attention kernels do
   // not overlap one another's compute), pbar is only touched by kernels that run one at a time
@@ -44,7 +48,7 @@ struct crystalkv {
   int* piece_ctr = nullptr;
   int cap_s = 0, pmax = 0;
   long long nA = 0;                // attention launches so far
-  std::vector<int> t_layer, par;   // per layer: time of the last step, current count buffer
+  std::vector<int> t_layer;        // per layer: time of the last step
   // LRFU launches are numbered; launch k uses scratch set k % NSETS and event k % EV_RING
   static constexpr int EV_RING = 32;
   cudaStream_t side = nullptr;
@@ -64,6 +68,9 @@ struct crystalkv {
   long long outJoined = -1;   // newest host step whose copy back the caller's stream has waited for
   long long nHost = 0;             // host-buffer steps so far
   __nv_bfloat16* dummy_out = nullptr;
+  int* io_rec = nullptr;           // staging for export / import of one head: records, rows, count
+  unsigned char* io_rows = nullptr;
+  int* io_n = nullptr;
   float* tab = nullptr;
   std::vector<void*> allocs;
   std::string err;
@@ -131,16 +138,15 @@ int dalloc(crystalkv_t* h, T** p, size_t count) {
   return CRYSTALKV_OK;
 }
 
-__global__ void init_free_stack_kernel(int* stack, int* top, long long slots_per_seq, int batch) {
-  const long long total = slots_per_seq * batch;
+__global__ void init_free_stack_kernel(int* stack, int* top, long long pages_per_seq, int batch) {
+  const long long total = pages_per_seq * batch;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
-    const long long r = i % slots_per_seq;
-    stack[i] = (int)(slots_per_seq - 1 - r);   // popping from the top hands out ascending slot ids
+    const long long r = i % pages_per_seq;
+    stack[i] = (int)(pages_per_seq - 1 - r);   // popping from the top hands out ascending page ids
   }
-  if (blockIdx.x == 0 && threadIdx.x < batch) top[threadIdx.x] = (int)slots_per_seq;
   if (blockIdx.x == 0)
-    for (int b = threadIdx.x; b < batch; b += blockDim.x) top[b] = (int)slots_per_seq;
+    for (int b = threadIdx.x; b < batch; b += blockDim.x) top[b] = (int)pages_per_seq;
 }
 
 __global__ void fill_int_kernel(int* p, long long n, int v) {
@@ -220,15 +226,14 @@ int check_unit(crystalkv_t* h, int layer, int seq, int head) {
   return CRYSTALKV_OK;
 }
 
-DecodeParams make_params(crystalkv_t* h, int layer, int set) {
+DecodeParams make_params(crystalkv_t* h, int layer) {
   DecodeParams p{};
   p.st = h->st;
-  (void)set;
+  p.plan = h->plans[layer];
+  p.done_ctr = h->done_ctr;
   p.sc.cap_s = h->cap_s;
   p.sc.pmax = h->pmax;
   p.sc.pbar = h->sc_pbar;
-  p.piece_ctr = h->piece_ctr;
-  p.parity = (int)(h->nA & 1);
   p.sc.partials = h->sc_partials[h->nA & 1];
   p.sc.ticket = h->sc_ticket[h->nA & 1];
   p.sc.logits = h->sc_logits[0];
@@ -236,14 +241,22 @@ DecodeParams make_params(crystalkv_t* h, int layer, int set) {
   h->nA++;
   p.layer = layer;
   p.G = h->G;
-  p.n_in = h->st.nbuf[h->par[layer]];
-  p.n_out = h->st.nbuf[h->par[layer] ^ 1];
   p.scale = h->cfg.sm_scale;
   p.scale_log2 = h->cfg.sm_scale * 1.44269504088896340736f;
   p.top_p = h->cfg.top_p;
   p.evict_every = h->cfg.evict_every;
   p.literal = h->cfg.literal_return;
+  p.plan_append = -1;
+  p.plan_warps = h->grid * NW;
+  p.plan_grid = h->grid;
   return p;
+}
+
+// Writes the launch plans of `count` layers from their heads' current lengths, on `s`.
+int replan(crystalkv_t* h, int layer0, int count, int append, int n_limit, cudaStream_t s) {
+  plan_kernel<<<count, NT, 0, s>>>(h->st, h->d_plans, layer0, append, n_limit, h->grid * NW, h->grid);
+  CK(h, cudaGetLastError());
+  return CRYSTALKV_OK;
 }
 
 // Makes `s` wait for every LRFU kernel launched so far.
@@ -255,9 +268,10 @@ int join_side(crystalkv_t* h, cudaStream_t s) {
   return CRYSTALKV_OK;
 }
 
-// One attention launch on `s` and, when Algorithm 1 runs, its LRFU launch on the internal stream.
+// One attention launch on `s` and its follow-up (Algorithm 1 when it runs, the heads' new lengths
+// and the layer's next plan) on the internal stream.
 int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
-  const bool track = p.track != 0;
+  const bool track = true;   // every launch has a follow-up that uses a scratch set
   const long long k = h->kF;
   if (track) {
     // launch k reuses the scratch of launch k - NSETS and continues the state its layer's
@@ -362,12 +376,19 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   h->U = c.batch * c.n_kv_heads;
   h->units = h->U * c.n_layers;
   // list positions per head: entries up to the largest budget plus those that arrive before the
-  // next eviction and the answer-stage tail, plus the spare; FullKV keeps every token
+  // next eviction and the answer-stage tail, plus the place of the next arrival; FullKV keeps
+  // every token.  Whole pages of 16.
   h->cap = evict ? c.max_budget + c.evict_every + c.max_answer_tokens + 1 : c.max_context + 1;
-  h->cap = (h->cap + GRP - 1) / GRP * GRP;   // whole 16-entry groups: a piece's slot ids are one aligned bulk copy
-  h->slots_per_seq = (long long)c.n_layers * c.n_kv_heads *
-                     (evict ? (long long)c.budget_per_head + c.evict_every + c.max_answer_tokens : (long long)c.max_context + 1);
-  if (h->slots_per_seq > 0x7fffffffLL) { g_create_err = "more than 2^31 slots per sequence"; delete h; return CRYSTALKV_EINVAL; }
+  h->cap = (h->cap + GRP - 1) / GRP * GRP;
+  // pages per sequence: the entries all heads may hold together (B_total, what arrives before an
+  // eviction, the answer tail, the hole), and one page per head for lists that end inside a page
+  {
+    const long long N = (long long)c.n_layers * c.n_kv_heads;
+    const long long per_head = evict ? (long long)c.budget_per_head + c.evict_every + c.max_answer_tokens + 1
+                                     : (long long)c.max_context + 1;
+    h->pages_per_seq = (N * per_head + GRP - 1) / GRP + N;
+  }
+  if (h->pages_per_seq > 0x7fffffffLL) { g_create_err = "more than 2^31 pages per sequence"; delete h; return CRYSTALKV_EINVAL; }
 
 #define CREATE_FAIL(code_)                    \
   do {                                        \
@@ -395,12 +416,11 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   cudaDeviceProp prop;
   CKC(cudaGetDeviceProperties(&prop, c.device));
   h->num_sms = prop.multiProcessorCount;
-  h->smem = RING_BYTES + (NW * STAGES + NW) * 8 + (size_t)(2 * h->U + 1) * sizeof(int);
+  // ring stages, one mbarrier per stage, every warp's queue of fetched pieces: the same for every
+  // handle (the attribute belongs to the function, so no handle may lower it under another)
+  h->smem = RING_BYTES + NW * STAGES * 8 + NW * FIFO * sizeof(int);
   int bps = 0;
-  // The attribute belongs to the function, not to the handle: it is set to the most any handle
-  // can ask for, so that a later, smaller handle does not lower it under an earlier one.
-  const size_t smem_max = RING_BYTES + (NW * STAGES + NW) * 8 + (size_t)(2 * MAX_UNITS_PER_CALL + 1) * sizeof(int);
-  CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
+  CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem));
   CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
   if (bps < 1) { h->err = "attention kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
   h->grid = h->num_sms * bps;
@@ -416,26 +436,43 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   for (cudaEvent_t& e : h->evF) CKC(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
 
   State& st = h->st;
-  st.batch = c.batch; st.L = c.n_layers; st.H = c.n_kv_heads; st.cap = h->cap;
-  st.slots_per_seq = h->slots_per_seq;
-  DA(&st.pool, (size_t)c.batch * h->slots_per_seq * SLOT_BYTES);
-  DA(&st.free_stack, (size_t)c.batch * h->slots_per_seq);
+  st.batch = c.batch; st.L = c.n_layers; st.H = c.n_kv_heads; st.cap = h->cap; st.capg = h->cap / GRP;
+  st.pages_per_seq = h->pages_per_seq;
+  DA(&st.pool, (size_t)c.batch * h->pages_per_seq * PAGE_BYTES);
+  DA(&st.free_stack, (size_t)c.batch * h->pages_per_seq);
   DA(&st.free_top, c.batch);
-  DA(&st.list_slot, (size_t)h->units * h->cap);
+  DA(&st.ptab, (size_t)h->units * st.capg);
   DA(&st.meta_pos, (size_t)h->units * h->cap);
   DA(&st.meta_tau, (size_t)h->units * h->cap);
   DA(&st.meta_crf, (size_t)h->units * h->cap);
-  DA(&st.nbuf[0], h->units);
-  DA(&st.nbuf[1], h->units);
+  DA(&st.n_cur, h->units);
+  DA(&st.hole, h->units);
+  DA(&st.npages, h->units);
   DA(&st.budget, h->units);
-  DA(&st.own, h->units);
+  // launch plans, one per layer: at most one piece per warp and one more per head
+  {
+    const int nWarps = h->grid * NW, pd_cap = nWarps + h->U;
+    int4* desc = nullptr; int2* wr = nullptr; int *npc = nullptr, *hdr = nullptr;
+    DA(&desc, (size_t)c.n_layers * pd_cap);
+    DA(&wr, (size_t)c.n_layers * nWarps);
+    DA(&npc, (size_t)c.n_layers * h->U);
+    DA(&hdr, (size_t)c.n_layers * 4);
+    CKC(cudaMemset(hdr, 0, (size_t)c.n_layers * 4 * sizeof(int)));
+    h->plans.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l)
+      h->plans[l] = Plan{desc + (size_t)l * pd_cap, wr + (size_t)l * nWarps, npc + (size_t)l * h->U, hdr + (size_t)l * 4};
+    DA(&h->d_plans, c.n_layers);
+    CKC(cudaMemcpy(h->d_plans, h->plans.data(), (size_t)c.n_layers * sizeof(Plan), cudaMemcpyHostToDevice));
+    DA(&h->done_ctr, 1);
+    CKC(cudaMemset(h->done_ctr, 0, sizeof(int)));
+  }
   DA(&h->tab, (size_t)c.max_context + 1);
   st.tab = h->tab;
   DA(&st.errword, 1);
   DA(&st.counters, 4);
   DA(&h->Asum, h->units);
   const int capgroups = (h->cap + GRP - 1) / GRP;
-  h->cap_s = evict ? ((h->cap + 3) & ~3) : 4;   // whole 128-byte lines of logit rows per unit
+  h->cap_s = evict ? h->cap : 4;   // whole 128-byte lines of logit rows per unit (cap is a multiple of 16)
   h->pmax = capgroups / GMIN + 2;
   for (int i = 0; i < NSETS; ++i) {
     DA(&h->sc_logits[i], (size_t)h->U * h->cap_s * QH);
@@ -452,6 +489,9 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
   for (int i = 0; i < crystalkv::HOST_RING; ++i) { DA(&h->dq[i], qn); DA(&h->dout[i], qn); DA(&h->dk[i], kn); DA(&h->dv[i], kn); }
   DA(&h->dummy_out, qn);
+  DA(&h->io_rec, (size_t)3 * h->cap);
+  DA(&h->io_rows, (size_t)2 * h->cap * ROW_BYTES);
+  DA(&h->io_n, 1);
 
   // lambda^D as fp32 from an fp64 pow; pow(0, 0) = 1 keeps same-step hits when lambda = 0
   {
@@ -459,17 +499,16 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     for (int D = 0; D <= c.max_context; ++D) tab[D] = (float)std::pow((double)c.lambda, (double)D);
     CKC(cudaMemcpy(h->tab, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice));
   }
-  init_free_stack_kernel<<<1024, 256>>>(st.free_stack, st.free_top, h->slots_per_seq, c.batch);
+  init_free_stack_kernel<<<1024, 256>>>(st.free_stack, st.free_top, h->pages_per_seq, c.batch);
   fill_int_kernel<<<256, 256>>>(st.budget, h->units, c.budget_per_head);
-  CKC(cudaMemset(st.nbuf[0], 0, (size_t)h->units * sizeof(int)));
-  CKC(cudaMemset(st.nbuf[1], 0, (size_t)h->units * sizeof(int)));
-  CKC(cudaMemset(st.own, 0, (size_t)h->units * sizeof(int)));
+  CKC(cudaMemset(st.n_cur, 0, (size_t)h->units * sizeof(int)));
+  CKC(cudaMemset(st.hole, 0, (size_t)h->units * sizeof(int)));
+  CKC(cudaMemset(st.npages, 0, (size_t)h->units * sizeof(int)));
   CKC(cudaMemset(st.errword, 0, sizeof(int)));
   CKC(cudaMemset(st.counters, 0, 4 * sizeof(unsigned long long)));
   CKC(cudaGetLastError());
   CKC(cudaDeviceSynchronize());
   h->t_layer.assign(c.n_layers, -1);
-  h->par.assign(c.n_layers, 0);
   h->lastF.assign(c.n_layers, -1);
   *out = h;
   return CRYSTALKV_OK;
@@ -511,10 +550,9 @@ static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* 
   if (h->t_layer[layer] >= 0) return fail(h, CRYSTALKV_ESTATE, "layer already prefilled");
   ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  rc = join_side(h, s);   // the insertion pops slots; no LRFU kernel may push or pop meanwhile
+  rc = join_side(h, s);   // the insertion takes pages; no LRFU kernel may take or return any meanwhile
   if (rc) return rc;
-  prefill_insert_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer,
-                                            static_cast<const __nv_bfloat16*>(k),
+  prefill_insert_kernel<<<h->U, NT, 0, s>>>(h->st, layer, static_cast<const __nv_bfloat16*>(k),
                                             static_cast<const __nv_bfloat16*>(v), P, W > 0 ? 1 : 0);
   CK(h, cudaGetLastError());
   if (evict) {
@@ -522,21 +560,29 @@ static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* 
     const size_t qn = (size_t)c.batch * c.n_q_heads * HD;
     for (int i = 0; i < passes; ++i) {
       // Algorithm 1 with the query of token t: steps 1-3 for every query, step 4 (down to the
-      // budget, freed slots back to the free list) after the last one
+      // budget, emptied pages back to the free list) after the last one
       const int t = P - passes + i;
-      DecodeParams p = make_params(h, layer, 0);
+      const bool last = i == passes - 1;
+      rc = replan(h, layer, 1, 0, last ? 0 : t + 1, s);   // a scoring pass over the first t + 1 entries
+      if (rc) return rc;
+      DecodeParams p = make_params(h, layer);
       p.q = static_cast<const __nv_bfloat16*>(q) + (size_t)i * qn;
       p.k_new = p.v_new = nullptr;
       p.out = out_window ? static_cast<__nv_bfloat16*>(out_window) + (size_t)i * qn : h->dummy_out;
       p.t = t;
       p.append = 0; p.track = 1; p.release = 1;
-      if (i < passes - 1) { p.n_limit = t + 1; p.hold = 1; }
+      if (!last) { p.n_limit = t + 1; p.hold = 1; }
+      else p.plan_append = 1;   // the layer's first decode step
+      h->prev_layer = -1;       // the plan kernel ahead writes what the attention kernel reads at once
       rc = launch_step(h, p, layer, s);
       if (rc) return rc;
     }
     rc = join_side(h, s);
     if (rc) return rc;
-    h->par[layer] ^= 1;
+  } else {
+    rc = replan(h, layer, 1, 1, 0, s);
+    if (rc) return rc;
+    h->prev_layer = -1;
   }
   h->t_layer[layer] = P - 1;
   return CRYSTALKV_OK;
@@ -569,16 +615,16 @@ int crystalkv_decode_step(crystalkv_t* h, int layer, const void* q, const void* 
     const int used = h->answer_steps / c.n_layers;
     if (used >= c.max_answer_tokens) return fail(h, CRYSTALKV_ESTATE, "max_answer_tokens reached");
   }
-  DecodeParams p = make_params(h, layer, 0);
+  DecodeParams p = make_params(h, layer);
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.k_new = static_cast<const __nv_bfloat16*>(k_new);
   p.v_new = static_cast<const __nv_bfloat16*>(v_new);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.t = t;
   p.append = 1; p.track = track ? 1 : 0; p.release = 0;
+  p.plan_append = 1;
   rc = launch_step(h, p, layer, static_cast<cudaStream_t>(stream));
   if (rc) return rc;
-  h->par[layer] ^= 1;
   h->t_layer[layer] = t;
   if (!track && c.mode == CRYSTALKV_MODE_EVICT) h->answer_steps++;
   return CRYSTALKV_OK;
@@ -660,14 +706,13 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   const crystalkv_config_t& c = h->cfg;
   if (c.mode != CRYSTALKV_MODE_EVICT) return fail(h, CRYSTALKV_ESTATE, "rebudget in FullKV mode");
   ON_DEVICE(h);
-  const int t_last = h->t_layer[0], par = h->par[0];
+  const int t_last = h->t_layer[0];
   if (t_last < 0) return fail(h, CRYSTALKV_ESTATE, "rebudget before prefill");
   for (int l = 1; l < c.n_layers; ++l)
-    if (h->t_layer[l] != t_last || h->par[l] != par) return fail(h, CRYSTALKV_ESTATE, "layers are at different time steps");
+    if (h->t_layer[l] != t_last) return fail(h, CRYSTALKV_ESTATE, "layers are at different time steps");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
-  int* n_cur = h->st.nbuf[par];
-  crf_sum_kernel<<<h->units, NT, 0, s>>>(h->st, n_cur, t_last, h->Asum);
+  crf_sum_kernel<<<h->units, NT, 0, s>>>(h->st, t_last, h->Asum);
   CK(h, cudaGetLastError());
   const int N = c.n_layers * c.n_kv_heads;
   const size_t sm = (size_t)N * (3 * sizeof(double) + sizeof(long long) + 2 * sizeof(int)) + (size_t)c.n_layers * 2 * sizeof(double);
@@ -676,10 +721,11 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   alg2_kernel<<<c.batch, NT, sm, s>>>(h->Asum, h->st.budget, c.n_layers, c.n_kv_heads, B_total, c.min_budget, c.max_budget);
   CK(h, cudaGetLastError());
   for (int l = 0; l < c.n_layers; ++l) {
-    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, n_cur, l, t_last, reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, l, t_last, reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
     CK(h, cudaGetLastError());
   }
-  return CRYSTALKV_OK;
+  // heads changed length: every layer's next decode step needs a new plan
+  return replan(h, 0, c.n_layers, 1, 0, s);
 }
 
 int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_t budget, void* stream) {
@@ -695,9 +741,9 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
   CK(h, cudaMemcpyAsync(h->st.budget + uid, &budget, sizeof(int), cudaMemcpyHostToDevice, s));
   CK(h, cudaStreamSynchronize(s));
   if (h->t_layer[layer] >= 0) {
-    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, h->st.nbuf[h->par[layer]], layer, h->t_layer[layer],
-                                      reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, layer, h->t_layer[layer], reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
     CK(h, cudaGetLastError());
+    return replan(h, layer, 1, 1, 0, s);
   }
   return CRYSTALKV_OK;
 }
@@ -712,38 +758,73 @@ int crystalkv_get_budgets(crystalkv_t* h, int32_t* out_host, void* stream) {
   return CRYSTALKV_OK;
 }
 
+// Copies one head's entries to the host, sorted by token position: records and, if asked for, rows.
+static int fetch_unit(crystalkv_t* h, int layer, int seq, int kv_head, std::vector<int32_t>& rec,
+                      std::vector<unsigned char>* krows, std::vector<unsigned char>* vrows, cudaStream_t s) {
+  const crystalkv_config_t& c = h->cfg;
+  if (int jr = join_side(h, s)) return jr;
+  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
+  export_unit_kernel<<<1, NT, 0, s>>>(h->st, uid, seq, h->io_rec, krows ? h->io_rows : nullptr,
+                                      krows ? h->io_rows + (size_t)h->cap * ROW_BYTES : nullptr, h->io_n);
+  CK(h, cudaGetLastError());
+  int n = 0;
+  CK(h, cudaMemcpyAsync(&n, h->io_n, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  std::vector<int32_t> raw((size_t)3 * n);
+  std::vector<unsigned char> kr, vr;
+  CK(h, cudaMemcpyAsync(raw.data(), h->io_rec, raw.size() * 4, cudaMemcpyDeviceToHost, s));
+  if (krows) {
+    kr.resize((size_t)n * ROW_BYTES); vr.resize((size_t)n * ROW_BYTES);
+    CK(h, cudaMemcpyAsync(kr.data(), h->io_rows, kr.size(), cudaMemcpyDeviceToHost, s));
+    CK(h, cudaMemcpyAsync(vr.data(), h->io_rows + (size_t)h->cap * ROW_BYTES, vr.size(), cudaMemcpyDeviceToHost, s));
+  }
+  CK(h, cudaStreamSynchronize(s));
+  std::vector<int> idx(n);
+  for (int i = 0; i < n; ++i) idx[i] = i;
+  std::sort(idx.begin(), idx.end(), [&](int a, int b) { return raw[3 * a] < raw[3 * b]; });
+  rec.resize((size_t)3 * n);
+  if (krows) { krows->resize((size_t)n * ROW_BYTES); vrows->resize((size_t)n * ROW_BYTES); }
+  for (int i = 0; i < n; ++i) {
+    std::memcpy(&rec[3 * i], &raw[3 * idx[i]], 12);
+    if (krows) {
+      std::memcpy(krows->data() + (size_t)i * ROW_BYTES, kr.data() + (size_t)idx[i] * ROW_BYTES, ROW_BYTES);
+      std::memcpy(vrows->data() + (size_t)i * ROW_BYTES, vr.data() + (size_t)idx[i] * ROW_BYTES, ROW_BYTES);
+    }
+  }
+  return CRYSTALKV_OK;
+}
+
 int crystalkv_export_state(crystalkv_t* h, int layer, int seq, int kv_head, int32_t* host_buf,
                            int32_t cap, int32_t* n_out, void* stream) {
   int rc = check_unit(h, layer, seq, kv_head);
   if (rc) return rc;
   if (!host_buf || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
   ON_DEVICE(h);
-  const crystalkv_config_t& c = h->cfg;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (int jr = join_side(h, s)) return jr;
-  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
-  int n = 0;
-  CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
-  CK(h, cudaStreamSynchronize(s));
+  std::vector<int32_t> rec;
+  rc = fetch_unit(h, layer, seq, kv_head, rec, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+  if (rc) return rc;
+  const int n = (int)(rec.size() / 3);
   *n_out = n;
   if (n > cap) return fail(h, CRYSTALKV_ESTATE, "buffer too small");
-  std::vector<int> pos(n), tau(n);
-  std::vector<float> crf(n);
-  const size_t mb = (size_t)uid * h->cap;
-  CK(h, cudaMemcpyAsync(pos.data(), h->st.meta_pos + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaMemcpyAsync(tau.data(), h->st.meta_tau + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaMemcpyAsync(crf.data(), h->st.meta_crf + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaStreamSynchronize(s));
-  std::vector<int> idx(n);
-  for (int i = 0; i < n; ++i) idx[i] = i;
-  std::sort(idx.begin(), idx.end(), [&](int a, int b) { return pos[a] < pos[b]; });
-  for (int i = 0; i < n; ++i) {
-    int32_t bits;
-    std::memcpy(&bits, &crf[idx[i]], 4);
-    host_buf[3 * i] = pos[idx[i]];
-    host_buf[3 * i + 1] = bits;
-    host_buf[3 * i + 2] = tau[idx[i]];
-  }
+  std::memcpy(host_buf, rec.data(), rec.size() * 4);
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_export_kv(crystalkv_t* h, int layer, int seq, int kv_head, void* k_rows_host, void* v_rows_host,
+                        int32_t cap, int32_t* n_out, void* stream) {
+  int rc = check_unit(h, layer, seq, kv_head);
+  if (rc) return rc;
+  if (!k_rows_host || !v_rows_host || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
+  ON_DEVICE(h);
+  std::vector<int32_t> rec;
+  std::vector<unsigned char> kr, vr;
+  rc = fetch_unit(h, layer, seq, kv_head, rec, &kr, &vr, static_cast<cudaStream_t>(stream));
+  if (rc) return rc;
+  const int n = (int)(rec.size() / 3);
+  *n_out = n;
+  if (n > cap) return fail(h, CRYSTALKV_ESTATE, "buffer too small");
+  std::memcpy(k_rows_host, kr.data(), kr.size());
+  std::memcpy(v_rows_host, vr.data(), vr.size());
   return CRYSTALKV_OK;
 }
 
@@ -753,54 +834,48 @@ int crystalkv_get_retained(crystalkv_t* h, int layer, int seq, int kv_head, int3
   if (rc) return rc;
   if (!pos_out_host || !n_out) return fail(h, CRYSTALKV_EINVAL, "null argument");
   ON_DEVICE(h);
-  const crystalkv_config_t& c = h->cfg;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (int jr = join_side(h, s)) return jr;
-  const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
-  int n = 0;
-  CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
-  CK(h, cudaStreamSynchronize(s));
+  std::vector<int32_t> rec;
+  rc = fetch_unit(h, layer, seq, kv_head, rec, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+  if (rc) return rc;
+  const int n = (int)(rec.size() / 3);
   *n_out = n;
   if (n > cap) return fail(h, CRYSTALKV_ESTATE, "buffer too small");
-  CK(h, cudaMemcpyAsync(pos_out_host, h->st.meta_pos + (size_t)uid * h->cap, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaStreamSynchronize(s));
-  std::sort(pos_out_host, pos_out_host + n);
+  for (int i = 0; i < n; ++i) pos_out_host[i] = rec[3 * i];
   return CRYSTALKV_OK;
 }
 
 int crystalkv_import_state(crystalkv_t* h, int layer, int seq, int kv_head, const int32_t* host_buf,
-                           int32_t n_rec, void* stream) {
+                           int32_t n_rec, const void* k_rows_host, const void* v_rows_host, int32_t budget,
+                           int32_t t, void* stream) {
   int rc = check_unit(h, layer, seq, kv_head);
   if (rc) return rc;
-  if (!host_buf || n_rec < 0) return fail(h, CRYSTALKV_EINVAL, "null argument");
-  ON_DEVICE(h);
+  if (!host_buf || !k_rows_host || !v_rows_host) return fail(h, CRYSTALKV_EINVAL, "null argument");
   const crystalkv_config_t& c = h->cfg;
+  if (n_rec < 1 || n_rec + 1 > h->cap) return fail(h, CRYSTALKV_EINVAL, "entry count outside [1, list capacity)");
+  if (budget < 0 || (c.mode == CRYSTALKV_MODE_EVICT && budget > c.max_budget)) return fail(h, CRYSTALKV_EINVAL, "budget outside [0, max_budget]");
+  if (t < 0 || t >= c.max_context) return fail(h, CRYSTALKV_EINVAL, "time outside [0, max_context)");
+  if (h->t_layer[layer] >= 0 && h->t_layer[layer] != t) return fail(h, CRYSTALKV_ESTATE, "the layer is at another time step");
+  for (int i = 0; i < n_rec; ++i)
+    if (host_buf[3 * i] < 0 || host_buf[3 * i] > t || host_buf[3 * i + 2] < 0 || host_buf[3 * i + 2] > t)
+      return fail(h, CRYSTALKV_EINVAL, "a record's position or last hit time lies after the layer's time");
+  ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
   const int uid = (seq * c.n_layers + layer) * c.n_kv_heads + kv_head;
-  int n = 0;
-  CK(h, cudaMemcpyAsync(&n, h->st.nbuf[h->par[layer]] + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
-  CK(h, cudaStreamSynchronize(s));
-  std::vector<int> pos(n), tau(n);
-  std::vector<float> crf(n);
-  const size_t mb = (size_t)uid * h->cap;
-  CK(h, cudaMemcpyAsync(pos.data(), h->st.meta_pos + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaMemcpyAsync(tau.data(), h->st.meta_tau + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaMemcpyAsync(crf.data(), h->st.meta_crf + mb, (size_t)n * 4, cudaMemcpyDeviceToHost, s));
-  CK(h, cudaStreamSynchronize(s));
-  std::vector<std::pair<int, int>> where(n);
-  for (int i = 0; i < n; ++i) where[i] = {pos[i], i};
-  std::sort(where.begin(), where.end());
-  for (int r = 0; r < n_rec; ++r) {
-    auto it = std::lower_bound(where.begin(), where.end(), std::make_pair((int)host_buf[3 * r], -1));
-    if (it == where.end() || it->first != host_buf[3 * r]) return fail(h, CRYSTALKV_ESTATE, "position not in the cache");
-    std::memcpy(&crf[it->second], &host_buf[3 * r + 1], 4);
-    tau[it->second] = host_buf[3 * r + 2];
+  CK(h, cudaMemcpyAsync(h->io_rec, host_buf, (size_t)n_rec * 12, cudaMemcpyHostToDevice, s));
+  CK(h, cudaMemcpyAsync(h->io_rows, k_rows_host, (size_t)n_rec * ROW_BYTES, cudaMemcpyHostToDevice, s));
+  CK(h, cudaMemcpyAsync(h->io_rows + (size_t)h->cap * ROW_BYTES, v_rows_host, (size_t)n_rec * ROW_BYTES, cudaMemcpyHostToDevice, s));
+  int b = budget;
+  if (b == 0) {
+    CK(h, cudaMemcpyAsync(&b, h->st.budget + uid, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CK(h, cudaStreamSynchronize(s));
   }
-  CK(h, cudaMemcpyAsync(h->st.meta_tau + mb, tau.data(), (size_t)n * 4, cudaMemcpyHostToDevice, s));
-  CK(h, cudaMemcpyAsync(h->st.meta_crf + mb, crf.data(), (size_t)n * 4, cudaMemcpyHostToDevice, s));
-  CK(h, cudaStreamSynchronize(s));
-  return CRYSTALKV_OK;
+  import_unit_kernel<<<1, NT, 0, s>>>(h->st, uid, seq, h->io_rec, h->io_rows, h->io_rows + (size_t)h->cap * ROW_BYTES, n_rec, b);
+  CK(h, cudaGetLastError());
+  CK(h, cudaStreamSynchronize(s));   // the host buffers and the staging area are free again
+  h->t_layer[layer] = t;
+  h->prev_layer = -1;
+  return replan(h, layer, 1, 1, 0, s);
 }
 
 int crystalkv_get_counters(crystalkv_t* h, uint64_t* entries_attended, uint64_t* hits,
@@ -827,14 +902,14 @@ int crystalkv_validate(crystalkv_t* h, void* stream) {
   ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (int jr = join_side(h, s)) return jr;
-  const long long total = (long long)c.batch * h->slots_per_seq;
+  const long long total = (long long)c.batch * h->pages_per_seq;
   int* seen = nullptr;
   CK(h, cudaMalloc(&seen, (size_t)(total + 2) * sizeof(int)));
   cudaError_t e = cudaMemsetAsync(seen, 0, (size_t)(total + 2) * sizeof(int), s);
   if (e == cudaSuccess) {
     mark_free_kernel<<<dim3(256, c.batch), 256, 0, s>>>(h->st, seen);
     for (int l = 0; l < c.n_layers; ++l)
-      mark_owned_kernel<<<h->U, 128, 0, s>>>(h->st, h->st.nbuf[h->par[l]], l, seen);
+      mark_owned_kernel<<<h->U, 128, 0, s>>>(h->st, l, seen);
     count_bad_kernel<<<1024, 256, 0, s>>>(seen, total, seen + total + 1);
     e = cudaGetLastError();
   }
@@ -844,16 +919,16 @@ int crystalkv_validate(crystalkv_t* h, void* stream) {
   cudaFree(seen);
   CK(h, e);
   if (res[0] || res[1])
-    return fail(h, CRYSTALKV_ECHECK, "slot ownership broken: " + std::to_string(res[0]) + " ids out of range, " +
-                                         std::to_string(res[1]) + " slots not owned exactly once");
+    return fail(h, CRYSTALKV_ECHECK, "page ownership broken: " + std::to_string(res[0]) + " ids or counts out of range, " +
+                                         std::to_string(res[1]) + " pages not owned exactly once");
   return CRYSTALKV_OK;
 }
 
-// ---- the slot-ownership check for callers that cannot allocate device memory
-// The per-slot counters live in this file-scope device array instead of a temporary from
-// cudaMalloc.  Every GPU that loads the library holds the array (8 MB) until the process exits.
-constexpr long long STATIC_SEEN_SLOTS = 1ll << 21;
-static __device__ __align__(256) int g_seen_static[STATIC_SEEN_SLOTS + 2];
+// ---- the page-ownership check for callers that cannot allocate device memory
+// The per-page counters live in this file-scope device array instead of a temporary from
+// cudaMalloc.  Every GPU that loads the library holds the array (512 KB) until the process exits.
+constexpr long long STATIC_SEEN_PAGES = 1ll << 17;
+static __device__ __align__(256) int g_seen_static[STATIC_SEEN_PAGES + 2];
 constexpr int STATIC_MAX_DEVICES = 64;
 static int* g_seen_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device ordinal
 static std::mutex g_seen_mu;                        // guards the look-up above
@@ -864,11 +939,11 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
   const crystalkv_config_t& c = h->cfg;
   for (int l = 0; l < c.n_layers; ++l)
     if (h->t_layer[l] < 0) return fail(h, CRYSTALKV_ESTATE, "validate before every layer is prefilled");
-  const long long total = (long long)c.batch * h->slots_per_seq;
-  if (total > STATIC_SEEN_SLOTS)
+  const long long total = (long long)c.batch * h->pages_per_seq;
+  if (total > STATIC_SEEN_PAGES)
     return fail(h, CRYSTALKV_EINVAL,
-                "crystalkv_validate_static: the handle has " + std::to_string(total) + " pool slots, the built-in "
-                "scratch covers " + std::to_string(STATIC_SEEN_SLOTS) + "; use crystalkv_validate");
+                "crystalkv_validate_static: the handle has " + std::to_string(total) + " pool pages, the built-in "
+                "scratch covers " + std::to_string(STATIC_SEEN_PAGES) + "; use crystalkv_validate");
   if (c.device >= STATIC_MAX_DEVICES) return fail(h, CRYSTALKV_EINVAL, "crystalkv_validate_static: device ordinal above 63");
   ON_DEVICE(h);
   int* seen = nullptr;
@@ -889,7 +964,7 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
   CK(h, cudaMemsetAsync(seen, 0, (size_t)(total + 2) * sizeof(int), s));
   mark_free_kernel<<<dim3(256, c.batch), 256, 0, s>>>(h->st, seen);
   for (int l = 0; l < c.n_layers; ++l)
-    mark_owned_kernel<<<h->U, 128, 0, s>>>(h->st, h->st.nbuf[h->par[l]], l, seen);
+    mark_owned_kernel<<<h->U, 128, 0, s>>>(h->st, l, seen);
   count_bad_kernel<<<1024, 256, 0, s>>>(seen, total, seen + total + 1);
   CK(h, cudaGetLastError());
   int res[2] = {0, 0};
@@ -897,8 +972,8 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
   CK(h, cudaStreamSynchronize(s));
   if (counts_out_host) { counts_out_host[0] = res[0]; counts_out_host[1] = res[1]; }
   if (res[0] || res[1])
-    return fail(h, CRYSTALKV_ECHECK, "slot ownership broken: " + std::to_string(res[0]) + " ids out of range, " +
-                                         std::to_string(res[1]) + " slots not owned exactly once");
+    return fail(h, CRYSTALKV_ECHECK, "page ownership broken: " + std::to_string(res[0]) + " ids or counts out of range, " +
+                                         std::to_string(res[1]) + " pages not owned exactly once");
   return CRYSTALKV_OK;
 }
 
@@ -920,11 +995,12 @@ int crystalkv_check(crystalkv_t* h, void* stream) {
   if (w == 0) return CRYSTALKV_OK;
   CK(h, cudaMemsetAsync(h->st.errword, 0, sizeof(int), s));
   std::string msg = "device error word:";
-  if (w & ERR_FREE_UNDERFLOW) msg += " free-list underflow;";
+  if (w & ERR_FREE_UNDERFLOW) msg += " free page list underflow;";
   if (w & ERR_OVER_EVICT) msg += " head further over its budget than the eviction period in a decode step;";
   if (w & ERR_CAPACITY) msg += " head list capacity exceeded;";
   if (w & ERR_NUCLEUS) msg += " top-p boundary not found;";
   if (w & ERR_COPY_TIMEOUT) msg += " a bulk copy into shared memory timed out;";
+  if (w & ERR_PLAN) msg += " a layer's launch plan did not fit the launch (or a head was empty);";
   return fail(h, CRYSTALKV_ECHECK, msg);
 }
 

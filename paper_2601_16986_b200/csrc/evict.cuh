@@ -1,7 +1,10 @@
-// Algorithm 1 step 4 as block-wide device routines: pick the k entries of a head that are
-// lowest under (CRF decayed to now, tau, position) and edit the head's slot list in place.
-// No K/V row is moved: a leaving entry's slot stays in the list past the live range as a
-// spare, and spares beyond one go back to the sequence's free list.
+// Algorithm 1 step 4 for the cases in which several entries leave a head at once (a prompt longer
+// than the budget, a budget that shrank, a buffered eviction cadence): pick the k entries lowest
+// under (CRF decayed to now, tau, position) by a radix select, then close the gaps they leave by
+// moving at most k entries from the end of the list into them (their rows and their metadata), so
+// that the list is dense again and the pages past its end can go back to the sequence's free
+// list.  (A decode step in which one entry leaves moves nothing: the arriving token of the next
+// step takes the leaver's place.)
 #pragma once
 #include "common.cuh"
 
@@ -27,37 +30,38 @@ __device__ __forceinline__ bool key_le(const Key96& a, const uint32_t* b) {
   return a.w[2] <= b[2];
 }
 
-// Moves entry `src` of a head into list position `dst` and leaves dst's slot at `src`.
-__device__ __forceinline__ void swap_into(const State& st, size_t mb, int dst, int src) {
-  const int freed = st.list_slot[mb + dst];
-  st.list_slot[mb + dst] = st.list_slot[mb + src];
-  st.meta_pos[mb + dst] = st.meta_pos[mb + src];
-  st.meta_tau[mb + dst] = st.meta_tau[mb + src];
-  st.meta_crf[mb + dst] = st.meta_crf[mb + src];
-  st.list_slot[mb + src] = freed;
+// Moves the entry at list position `src` of a head to position `dst` (one warp: lane c carries
+// chunk c of the 512-byte row, which sits at a different place in the two pages' layouts).
+__device__ __forceinline__ void move_entry(const State& st, int uid, int seq, size_t mb, int dst, int src, int lane) {
+  const uint4 v = *reinterpret_cast<const uint4*>(entry_chunk(st, uid, seq, src, lane));
+  *reinterpret_cast<uint4*>(entry_chunk(st, uid, seq, dst, lane)) = v;
+  if (lane == 0) {
+    st.meta_pos[mb + dst] = st.meta_pos[mb + src];
+    st.meta_tau[mb + dst] = st.meta_tau[mb + src];
+    st.meta_crf[mb + dst] = st.meta_crf[mb + src];
+  }
 }
 
-// The head's spares beyond the one at list position n_new (the freed slots and the spares it
-// held before) return to the sequence's free list.  Only called from launches in which no head
-// pops a slot.
-__device__ __forceinline__ void release_spares(const State& st, size_t mb, int uid, int seq, int n_new,
-                                               int* s_base) {
-  const int cnt = st.own[uid] - (n_new + 1);
+// The pages a head owns beyond those that back list positions 0 .. n_new return to the
+// sequence's free list.  Only called from launches in which no head takes a page.
+__device__ __forceinline__ void release_pages(const State& st, int uid, int seq, int n_new, int* s_base) {
+  const int need = n_new / GRP + 1;   // position n_new (the hole) stays backed
+  const int have = st.npages[uid];
+  const int cnt = have - need;
   if (cnt <= 0) return;
   if (threadIdx.x == 0) *s_base = atomicAdd(&st.free_top[seq], cnt);
   __syncthreads();
   const int base = *s_base;
-  int* stack = st.free_stack + (size_t)seq * st.slots_per_seq;
-  for (int r = threadIdx.x; r < cnt; r += NT) stack[base + r] = st.list_slot[mb + n_new + 1 + r];
+  int* stack = st.free_stack + (size_t)seq * st.pages_per_seq;
+  for (int r = threadIdx.x; r < cnt; r += NT) stack[base + r] = st.ptab[(size_t)uid * st.capg + need + r];
   __syncthreads();
-  if (threadIdx.x == 0) st.own[uid] = n_new + 1;
+  if (threadIdx.x == 0) st.npages[uid] = need;
 }
 
-// Removes the k lowest entries (1 <= k < n) of head `uid` at time t.  With `release` the head
-// must own a spare at list position n (true between steps and after prompt insertion).  `sh` is >= 1.2 KB (300 ints) of
-// shared scratch, `tmp` a global int scratch of >= n words.  All NT threads call it.
-__device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n, int k, int t,
-                           bool release, int* sh, int* tmp) {
+// Removes the k lowest entries (1 <= k < n) of head `uid` at time t; the head's n entries must be
+// dense (list positions 0 .. n-1).  `sh` is >= 1.2 KB (300 ints) of shared scratch, `tmp` a global
+// int scratch of >= n words.  All NT threads call it.
+__device__ void evict_many(const State& st, int uid, int seq, int n, int k, int t, bool release, int* sh, int* tmp) {
   const size_t mb = (size_t)uid * st.cap;
   int* hist = sh;             // 256
   int* s_kw = sh + 256;       // 3 words of the k-th key
@@ -121,33 +125,36 @@ __device__ void evict_many(const State& st, int* n_out, int uid, int seq, int n,
   }
   const uint32_t kth[3] = {(uint32_t)s_kw[0], (uint32_t)s_kw[1], (uint32_t)s_kw[2]};
   const int nk = n - k;
-  // holes: leaving entries inside the surviving range [0, nk)
-  int run = 0;
+  // gaps: leaving entries inside the surviving range [0, nk)
+  int gaps = 0;
   for (int base = 0; base < nk; base += NT) {
     const int i = base + tid;
     const int flag = (i < nk) && key_le(entry_key(st, mb, i, t), kth);
     int tot;
     const int r = block_excl_scan(flag, red, tot);
-    if (flag) tmp[run + r] = i;
-    run += tot;
+    if (flag) tmp[gaps + r] = i;
+    gaps += tot;
   }
-  __syncthreads();
-  // movers: staying entries in the tail [nk, n) fill the holes in order
-  run = 0;
+  // movers: staying entries in the tail [nk, n), as many as there are gaps
+  int movers = 0;
   for (int base = nk; base < n; base += NT) {
     const int i = base + tid;
     const int flag = (i < n) && !key_le(entry_key(st, mb, i, t), kth);
     int tot;
     const int r = block_excl_scan(flag, red, tot);
-    if (flag) swap_into(st, mb, tmp[run + r], i);
-    run += tot;
+    if (flag) tmp[gaps + movers + r] = i;
+    movers += tot;
   }
   __syncthreads();
+  // every mover fills one gap, in order; rows and metadata travel together
+  for (int j = tid >> 5; j < min(gaps, movers); j += NW) move_entry(st, uid, seq, mb, tmp[j], tmp[gaps + j], tid & 31);
+  __syncthreads();
   if (tid == 0) {
-    n_out[uid] = nk;
+    st.n_cur[uid] = nk;
+    st.hole[uid] = nk;
     atomicAdd(&st.counters[2], (unsigned long long)k);
   }
-  if (release) release_spares(st, mb, uid, seq, nk, s_krem);
+  if (release) release_pages(st, uid, seq, nk, s_krem);
 }
 
 }  // namespace ckv

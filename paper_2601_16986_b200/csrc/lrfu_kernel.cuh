@@ -10,12 +10,16 @@
 //   step 2-3 hits: CRF <- lambda^(t - tau) CRF + 1, tau <- t; misses only get the decayed
 //            CRF_temp, which is not stored;
 //   step 4   the entries lowest under (CRF_temp, tau, position) leave until the head is
-//            within its budget; the freed slot is reused in place.
+//            within its budget; the place of a single leaver becomes the head's hole, which
+//            the next arriving token fills: nothing is moved.
+// A launch without Algorithm 1 (answer stage, full-cache mode) only lets every head keep its new
+// entry.  Either way the CTA that finishes last writes the layer's next launch plan (plan.cuh).
 // The mass walk uses 2^-40 fixed-point integers so it is exact and order independent; the
 // threshold is relative to the integer total, so a common factor on pbar changes nothing.
 #pragma once
 #include "common.cuh"
 #include "evict.cuh"
+#include "plan.cuh"
 
 namespace ckv {
 
@@ -37,10 +41,11 @@ struct LrfuSmem {
   int ncand;
   int star;
   int eq[NW];
-  int amin[NW * 5];
-  int last[4];   // slot, position, tau, CRF bits of list position n-1 after the update
+  int amin[NW * 4];
   int ev[320];
+  int is_last;
 };
+static_assert(sizeof(LrfuSmem) >= (MAX_UNITS_PER_CALL + 1) * sizeof(int) + 321 * sizeof(int), "the planner's prefix sums reuse this memory");
 
 // Loads the compiler must leave where they are written: the kernel is bound by the latency of
 // its dependent global reads (several microseconds each while the attention kernel saturates
@@ -105,7 +110,7 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   float pmr[R];
   // stored state of this thread's entries, requested as soon as the logits are consumed so that
   // the reads complete under the threshold search (EPT == FRONT only)
-  int pos_r[R], tau_r[R], slot_last = 0;
+  int pos_r[R], tau_r[R];
   float crf_r[R];
   if (EPT == FRONT) {
 #pragma unroll
@@ -123,7 +128,6 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       tau_r[k] = ld_i32(st.meta_tau + i);
       crf_r[k] = ld_f32(st.meta_crf + i);
     }
-    if (tid == (n - 1) % NT) slot_last = ld_i32(st.list_slot + mb + n - 1);   // the owner of the last entry
     // The logit rows are dead now (every thread holds its own in registers since before the
     // kernel learnt n, and nothing reads them again): drop their L2 lines instead of letting
     // them be written back to DRAM later.  Four 32-byte rows share a 128-byte line; units start
@@ -435,17 +439,7 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
 #pragma unroll
     for (int k = 0; k < R; ++k) {
       const int i = tid + k * NT;
-      if (i < n) {
-        const int nh = nhit;
-        update(i, pmr[k], pos_r[k], tau_r[k], crf_r[k], dec_r[k]);
-        if (i == n - 1) {   // what list position n-1 holds after this step, for the in-place swap
-          const bool hit = nhit != nh;
-          sh.last[0] = slot_last;
-          sh.last[1] = pos_r[k];
-          sh.last[2] = hit ? p.t : tau_r[k];
-          sh.last[3] = __float_as_int(hit ? __fadd_rn(__fmul_rn(dec_r[k], crf_r[k]), 1.0f) : crf_r[k]);
-        }
-      }
+      if (i < n) update(i, pmr[k], pos_r[k], tau_r[k], crf_r[k], dec_r[k]);
     }
   } else {
     for (int i = tid; i < n; i += NT) {
@@ -457,51 +451,38 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   if (lane == 0 && nhit) atomicAdd(&st.counters[1], (unsigned long long)nhit);
   int n_after = n;
   if (k_evict == 1) {
-    // block argmin of (CRF_temp, tau, pos); every thread asks for the slot of its own candidate
-    // now, so the winner's is at hand when the reduction ends
-    int bslot = (EPT == FRONT && bidx >= 0) ? ld_i32(st.list_slot + mb + bidx) : 0;
+    // block argmin of (CRF_temp, tau, pos)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const uint32_t o0 = __shfl_xor_sync(0xffffffffu, bk0, o), o1 = __shfl_xor_sync(0xffffffffu, bk1, o),
                      o2 = __shfl_xor_sync(0xffffffffu, bk2, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bidx, o), os = __shfl_xor_sync(0xffffffffu, bslot, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bidx, o);
       const bool less = (o0 != bk0) ? (o0 < bk0) : ((o1 != bk1) ? (o1 < bk1) : (o2 < bk2));
-      if (less) { bk0 = o0; bk1 = o1; bk2 = o2; bidx = oi; bslot = os; }
+      if (less) { bk0 = o0; bk1 = o1; bk2 = o2; bidx = oi; }
     }
-    if (lane == 0) { sh.amin[w * 5] = (int)bk0; sh.amin[w * 5 + 1] = (int)bk1; sh.amin[w * 5 + 2] = (int)bk2; sh.amin[w * 5 + 3] = bidx; sh.amin[w * 5 + 4] = bslot; }
-    __syncthreads();   // also orders every CRF/tau store above before the swap below
+    if (lane == 0) { sh.amin[w * 4] = (int)bk0; sh.amin[w * 4 + 1] = (int)bk1; sh.amin[w * 4 + 2] = (int)bk2; sh.amin[w * 4 + 3] = bidx; }
+    __syncthreads();
     if (tid == 0) {
       uint32_t a0 = (uint32_t)sh.amin[0], a1 = (uint32_t)sh.amin[1], a2 = (uint32_t)sh.amin[2];
-      int ai = sh.amin[3], as = sh.amin[4];
+      int ai = sh.amin[3];
       for (int x = 1; x < NW; ++x) {
-        const uint32_t o0 = (uint32_t)sh.amin[x * 5], o1 = (uint32_t)sh.amin[x * 5 + 1], o2 = (uint32_t)sh.amin[x * 5 + 2];
+        const uint32_t o0 = (uint32_t)sh.amin[x * 4], o1 = (uint32_t)sh.amin[x * 4 + 1], o2 = (uint32_t)sh.amin[x * 4 + 2];
         const bool less = (o0 != a0) ? (o0 < a0) : ((o1 != a1) ? (o1 < a1) : (o2 < a2));
-        if (less) { a0 = o0; a1 = o1; a2 = o2; ai = sh.amin[x * 5 + 3]; as = sh.amin[x * 5 + 4]; }
+        if (less) { a0 = o0; a1 = o1; a2 = o2; ai = sh.amin[x * 4 + 3]; }
       }
-      // the leaving entry's slot becomes the head's spare at position n-1
-      if (ai != n - 1) {
-        if (EPT == FRONT) {   // everything needed is already here: stores only
-          st.list_slot[mb + ai] = sh.last[0];
-          st.meta_pos[mb + ai] = sh.last[1];
-          st.meta_tau[mb + ai] = sh.last[2];
-          st.meta_crf[mb + ai] = __int_as_float(sh.last[3]);
-          st.list_slot[mb + n - 1] = as;
-        } else {
-          swap_into(st, mb, ai, n - 1);
-        }
-      }
-      p.n_out[uid] = n - 1;
+      // the leaving entry's place is where the next arriving token is written
+      st.hole[uid] = ai;
+      st.n_cur[uid] = n - 1;
       atomicAdd(&st.counters[2], 1ull);
     }
     n_after = n - 1;
   } else if (k_evict > 1) {
     __syncthreads();
     if (p.append && k_evict > p.evict_every && tid == 0) atomicOr(st.errword, ERR_OVER_EVICT);
-    evict_many(st, p.n_out, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh.ev,
-               reinterpret_cast<int*>(pbar));
+    evict_many(st, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh.ev, reinterpret_cast<int*>(pbar));
     n_after = n - min(k_evict, n - 1);
   }
-  if (n_after == n && tid == 0 && !p.hold) keep_and_refill(st, p.n_out, uid, seq, n, p.append != 0);
+  if (n_after == n && tid == 0 && !p.hold) keep_all(st, uid, seq, n, p.append != 0);
 }
 
 template <int G>
@@ -512,36 +493,53 @@ __global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
   const int uid = (seq * st.L + p.layer) * st.H + head;
   // one batch of requests: the length, the budget, the softmax reference, and the logit rows the
   // common path needs (requested for a full thread's worth, clamped to the scratch)
-  int n_raw = ld_i32(p.n_in + uid);
+  int n_raw = ld_i32(st.n_cur + uid);
   if (p.n_limit > 0) n_raw = min(n_raw, p.n_limit);
-  Front<G> fr;
-  fr.budget = ld_i32(st.budget + uid);
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    fr.m[g] = ld_f32(p.sc.mfin + u * (2 * QH) + g);
-    fr.l[g] = ld_f32(p.sc.mfin + u * (2 * QH) + QH + g);
-  }
-  {
-    const float* S = p.sc.logits + (size_t)u * p.sc.cap_s * QH;
-#pragma unroll
-    for (int k = 0; k < FRONT; ++k) {
-      const int i = min((int)threadIdx.x + k * NT, p.sc.cap_s - 1);
-      fr.ra[k] = ld_f32x4(S + (size_t)i * QH);
-      fr.rb[k] = (G > 4) ? ld_f32x4(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-  }
   const int n = n_raw + p.append;
-  if (n <= 0) {
-    if (threadIdx.x == 0 && !p.hold) p.n_out[uid] = 0;
-    return;
+  if (p.track) {
+    Front<G> fr;
+    fr.budget = ld_i32(st.budget + uid);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      fr.m[g] = ld_f32(p.sc.mfin + u * (2 * QH) + g);
+      fr.l[g] = ld_f32(p.sc.mfin + u * (2 * QH) + QH + g);
+    }
+    {
+      const float* S = p.sc.logits + (size_t)u * p.sc.cap_s * QH;
+#pragma unroll
+      for (int k = 0; k < FRONT; ++k) {
+        const int i = min((int)threadIdx.x + k * NT, p.sc.cap_s - 1);
+        fr.ra[k] = ld_f32x4(S + (size_t)i * QH);
+        fr.rb[k] = (G > 4) ? ld_f32x4(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    if (n <= 0) {
+      if (threadIdx.x == 0 && !p.hold) { st.n_cur[uid] = 0; st.hole[uid] = 0; }
+    } else if (p.literal && n < fr.budget) {   // Algorithm 1's first line as printed: nothing runs below the budget
+      if (threadIdx.x == 0 && !p.hold) keep_all(st, uid, seq, n, p.append != 0);
+    } else if (n <= FRONT * NT) {
+      lrfu_unit<G, FRONT>(p, u, uid, seq, n, sh, fr);
+    } else if (n <= 17 * NT) {
+      lrfu_unit<G, 17>(p, u, uid, seq, n, sh, fr);
+    } else {
+      lrfu_unit<G, 0>(p, u, uid, seq, n, sh, fr);
+    }
+  } else if (threadIdx.x == 0) {
+    keep_all(st, uid, seq, n, p.append != 0);   // no Algorithm 1: the head keeps its new entry
   }
-  if (p.literal && n < fr.budget) {   // Algorithm 1's first line as printed: nothing runs below the budget
-    if (threadIdx.x == 0 && !p.hold) keep_and_refill(st, p.n_out, uid, seq, n, p.append != 0);
-    return;
+  if (threadIdx.x == 0) atomicAdd(&st.counters[0], (unsigned long long)max(n, 0));
+  if (p.plan_append < 0) return;
+  // ---- the CTA that finishes last knows every head's new length: it writes the layer's next plan
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const int done = atomicAdd(p.done_ctr, 1);
+    sh.is_last = (done == (int)gridDim.x - 1);
+    if (sh.is_last) { *p.done_ctr = 0; __threadfence(); }
   }
-  if (n <= FRONT * NT) lrfu_unit<G, FRONT>(p, u, uid, seq, n, sh, fr);
-  else if (n <= 17 * NT) lrfu_unit<G, 17>(p, u, uid, seq, n, sh, fr);
-  else lrfu_unit<G, 0>(p, u, uid, seq, n, sh, fr);
+  __syncthreads();
+  if (!sh.is_last) return;
+  write_plan(st, p.plan, p.layer, p.plan_append, 0, p.plan_warps, p.plan_grid, reinterpret_cast<int*>(&sh), sh.ev);
 }
 
 }  // namespace ckv

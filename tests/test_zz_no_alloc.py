@@ -87,10 +87,10 @@ def test_static_check_after_a_larger_handle_used_the_array():
 
 
 def test_static_check_refuses_a_handle_beyond_its_array():
-    """2**21 slots is the limit; one sequence more than fits is refused with EINVAL and a
-    message that names the limit, and nothing is launched."""
+    """2**17 pool pages (16 entries each) is the limit; a handle with more is refused with EINVAL
+    and a message that names the limit, and nothing is launched."""
     kv = CrystalKV(Config(n_layers=8, n_q_heads=8, n_kv_heads=8, batch=17, budget_per_head=2047,
-                          max_context=64))       # 17 * 8 * 8 * 2048 slots > 2**21
+                          max_context=64))       # 17 * (8 * 8 * 2049 / 16 + 64) pages > 2**17
     pk = torch.zeros(17, 4, 8, 128, dtype=torch.bfloat16, device="cuda")
     q = torch.zeros(17, 8, 128, dtype=torch.bfloat16, device="cuda")
     for l in range(8):
@@ -98,7 +98,7 @@ def test_static_check_refuses_a_handle_beyond_its_array():
     counts = np.full(2, -1, dtype=np.int32)
     rc = kv.lib.crystalkv_validate_static(kv._h, counts.ctypes.data_as(C.c_void_p), None)
     assert rc == -1
-    assert b"2097152" in kv.lib.crystalkv_last_error(kv._h)
+    assert b"131072" in kv.lib.crystalkv_last_error(kv._h)
     assert tuple(counts) == (-1, -1)
     assert _verdict(kv.validate)[0] == 0         # the allocating entry point still serves it
     kv.close()
