@@ -54,6 +54,7 @@ typedef struct {
     double tie_eps; /* relative window for the tie log (1e-6) */
     int32_t evict_every;    /* m: step 4 runs once a head is m entries over its budget (0, 1: every step) */
     int32_t literal_return; /* 1: Algorithm 1's first line taken literally (nothing runs while Len(K) < B) */
+    float budget_ratio;     /* r > 0: budgets follow the context, r x tokens per head on average (0: fixed) */
 } okv_config;
 
 typedef struct {
@@ -369,6 +370,23 @@ static void lrfu_pass(okv *o, int seq, int layer, int head, const uint16_t *q, i
     lrfu_pass_unit(o, unit_of(o, seq, layer, head), seq, layer, head, q, t, track, hold, y, 0);
 }
 
+/*
+ * Ratio budgets (Section 6.1 and Table 1's "Ratio-10 %" rows: a budget of 10 % of the tokens,
+ * 935 entries per head of 9 350 tokens, 1 870 of 18 700).  Reading: the average budget per head
+ * after `tokens` tokens is floor(r * tokens), evaluated in fp64 from the fp32 ratio, kept
+ * between max(1, min_budget) and budget_per_head (which sizes the storage); it is applied when
+ * the prompt is loaded (uniformly) and as Algorithm 2's B_total at every reallocation.
+ */
+static int32_t ratio_budget(const okv_config *c, int tokens) {
+    int64_t b = (int64_t)floor((double)c->budget_ratio * (double)tokens);
+    int64_t lo = c->min_budget > 1 ? c->min_budget : 1;
+    if (b < lo) b = lo;
+    if (b > c->budget_per_head) b = c->budget_per_head;
+    return (int32_t)b;
+}
+
+int32_t okv_ratio_budget(okv *o, int tokens) { return ratio_budget(&o->c, tokens); }
+
 /* ------------------------------------------------------------------ lifecycle */
 
 okv *okv_create(const okv_config *c) {
@@ -417,6 +435,7 @@ int okv_prefill(okv *o, int layer, const uint16_t *k, const uint16_t *v, const u
     for (int b = 0; b < c->batch; ++b)
         for (int h = 0; h < H; ++h) {
             okv_unit *u = unit_of(o, b, layer, h);
+            if (c->budget_ratio > 0.0f) u->budget = ratio_budget(c, P);
             for (int i = 0; i < P; ++i) {
                 size_t off = (((size_t)b * P + i) * H + h) * d;
                 unit_append(o, u, i, k + off, v + off, 0.0f, P - 1);
@@ -447,6 +466,7 @@ int okv_prefill_window(okv *o, int layer, const uint16_t *k, const uint16_t *v, 
     for (int b = 0; b < c->batch; ++b)
         for (int h = 0; h < H; ++h) {
             okv_unit *u = unit_of(o, b, layer, h);
+            if (c->budget_ratio > 0.0f) u->budget = ratio_budget(c, P);
             for (int i = 0; i < P; ++i) {
                 size_t off = (((size_t)b * P + i) * H + h) * d;
                 unit_append(o, u, i, k + off, v + off, 0.0f, i);
@@ -611,6 +631,7 @@ int okv_rebudget(okv *o) {
         if (o->t_layer[l] != t_last || t_last < 0) return OKV_ERR;
     if (c->mode != OKV_MODE_EVICT) return OKV_ERR;
     int64_t B_total = (int64_t)c->budget_per_head * L * H;
+    if (c->budget_ratio > 0.0f) B_total = (int64_t)ratio_budget(c, t_last + 1) * L * H;
 #pragma omp parallel for schedule(dynamic)
     for (int b = 0; b < c->batch; ++b) {
         double *A = (double *)malloc((size_t)L * H * sizeof(double));

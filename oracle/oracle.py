@@ -24,7 +24,7 @@ class _Cfg(C.Structure):
                 ("min_budget", C.c_int32), ("max_budget", C.c_int32), ("max_context", C.c_int32),
                 ("mode", C.c_int32), ("top_p", C.c_float), ("lam", C.c_float),
                 ("sm_scale", C.c_float), ("tie_eps", C.c_double),
-                ("evict_every", C.c_int32), ("literal_return", C.c_int32)]
+                ("evict_every", C.c_int32), ("literal_return", C.c_int32), ("budget_ratio", C.c_float)]
 
 
 @dataclass
@@ -45,6 +45,7 @@ class OracleConfig:
     tie_eps: float = 1e-6
     evict_every: int = 1         # m: evict once a head is m entries over its budget
     literal_return: int = 0      # 1: no tracking while a head is below its budget (Algorithm 1, first line)
+    budget_ratio: float = 0.0    # r > 0: the average budget per head follows the context, floor(r * tokens)
 
 
 _lib = None
@@ -70,6 +71,7 @@ def _load():
         lib.okv_export_state.argtypes = [vp, i32, i32, i32, vp, i32]
         lib.okv_import_state.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp]
         lib.okv_replay_unit.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32]
+        lib.okv_ratio_budget.argtypes = [vp, i32]
         lib.okv_tie_count.argtypes = [vp]
         lib.okv_get_ties.argtypes = [vp, vp, i32]
         lib.okv_clear_ties.argtypes = [vp]
@@ -137,7 +139,8 @@ class Oracle:
         max_b = cfg.max_budget or cfg.budget_per_head * cfg.n_layers * cfg.n_kv_heads
         self._c = _Cfg(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.batch,
                        cfg.budget_per_head, cfg.min_budget, max_b, cfg.max_context, cfg.mode,
-                       cfg.top_p, cfg.lam, cfg.sm_scale, cfg.tie_eps, cfg.evict_every, cfg.literal_return)
+                       cfg.top_p, cfg.lam, cfg.sm_scale, cfg.tie_eps, cfg.evict_every, cfg.literal_return,
+                       cfg.budget_ratio)
         self._h = lib.okv_create(C.byref(self._c))
         if not self._h:
             raise ValueError("oracle: bad config")
@@ -207,6 +210,10 @@ class Oracle:
 
     def time(self, layer) -> int:
         return self._lib.okv_time(self._h, layer)
+
+    def ratio_budget(self, tokens: int) -> int:
+        """Average budget per head after `tokens` tokens under the configured ratio."""
+        return int(self._lib.okv_ratio_budget(self._h, int(tokens)))
 
     def export_state(self, layer, seq, head) -> np.ndarray:
         """-> int32 [n,3] rows (pos, crf bits, tau) sorted by pos."""

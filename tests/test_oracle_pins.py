@@ -747,3 +747,42 @@ def test_replay_of_one_head_follows_the_run_and_a_flip_moves_one_entry():
                          v[0, P - 1:P, h].contiguous(), np.zeros(1, dtype=np.int32), append_first=False)
     assert (got == o2.export_state(0, 0, h)).all()
     o.close(); o2.close()
+
+
+# ------------------------------------------------------------ ratio budgets (Table 1's "Ratio-10 %" rows)
+def test_ratio_budget_is_table1_closed_form_and_is_conserved():
+    """A 10 % ratio gives Table 1's budgets (935 entries per head of 9 350 tokens, 1 870 of 18 700);
+    under a ratio the budgets of a sequence sum, after every reallocation, to that budget times
+    the number of heads, start from the prompt's share, and never shrink as the context grows."""
+    rows = [l.split() for l in open(os.path.join(GOLD, "table1_hbm_saving.txt")) if l[0] != "#"]
+    w = tiny(n_layers=2, n_q_heads=4, n_kv_heads=2, batch=2, prompt=24, think_steps=64, budget_per_head=4096,
+             seed=33, outlier="perhead", outlier_lo=0.05, outlier_hi=0.4)
+    o = make_oracle(w, budget_ratio=0.1, min_budget=1, max_budget=4096)
+    for budget, tokens, saving in rows:
+        if float(saving) == 90.0:
+            assert o.ratio_budget(int(tokens)) == int(budget) == int(tokens) // 10
+    o.close()
+    o = make_oracle(w, budget_ratio=0.25, min_budget=2, max_budget=64, budget_per_head=20)
+    for l in range(w.n_layers):
+        k, v = w.prompt_kv(l)
+        o.prefill(l, k, v, w.queries(l, [w.prompt - 1])[:, 0])
+    assert (o.get_budgets() == 6).all()                       # floor(0.25 * 24)
+    for l in range(w.n_layers):
+        assert all(len(o.get_retained(l, b, h)) == 6 for b in range(2) for h in range(2))
+    prev_total = 6 * 4
+    for t in range(w.prompt, w.prompt + w.think_steps):
+        for l in range(w.n_layers):
+            o.decode_step(l, *w.step_inputs(l, t))
+        if (t - w.prompt + 1) % 8 == 0:
+            o.rebudget()
+            B = o.get_budgets()
+            want = min(20, (t + 1) // 4)                       # floor(0.25 * tokens), capped by budget_per_head
+            assert (B.reshape(2, -1).sum(axis=1) == want * 4).all()
+            assert want * 4 >= prev_total and B.min() >= 2
+            prev_total = want * 4
+            for b in range(2):
+                for l in range(w.n_layers):
+                    for h in range(2):
+                        assert len(o.get_retained(l, b, h)) <= B[b, l, h]
+    assert prev_total == 20 * 4 and (o.get_budgets() != 20).any()
+    o.close()
