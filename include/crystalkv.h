@@ -69,6 +69,11 @@ typedef struct {
                               removes all of them in one call (k = m); 0 or 1 = every step.  At most 4096. */
   int32_t literal_return;  /* 1: Algorithm 1's first line as printed: while Len(K) < B of a head nothing
                               of the algorithm runs for it (no hit mask, no CRF update); 0 = track always */
+  float budget_ratio;      /* r > 0: ratio budgets (Section 6.1, Table 1's "Ratio-10 %" rows): the average budget
+                              per head follows the context, floor(r * tokens) kept within [max(1, min_budget),
+                              budget_per_head]; set uniformly when the prompt is loaded and used as Algorithm 2's
+                              B_total (times L * H) at every reallocation.  budget_per_head still sizes the
+                              storage.  0 = fixed budgets */
 } crystalkv_config_t;
 
 /*
@@ -86,8 +91,10 @@ int crystalkv_destroy(crystalkv_t* h);
  * Algorithm 1 pass with Q^last at t = P-1, so CRF/tau are seeded and heads whose
  * prompt exceeds their budget are evicted down to it.
  *   k, v   dev  [batch][P][H][128]     q_last dev [batch][Hq][128] (query of token P-1)
- * P must satisfy 1 <= P <= budget_per_head + max_answer_tokens (evict mode) or
- * P < max_context (FullKV mode).  Errors: EINVAL; ESTATE if the layer was prefilled.
+ * A prompt longer than the budget is scored from k and q_last as they are, and only the rows
+ * of the entries Algorithm 1 retains are stored, so the pool never holds more than the budget.
+ * P must satisfy 1 <= P < max_context and P <= max_budget + evict_every + max_answer_tokens (the
+ * heads' list capacity).  Errors: EINVAL; ESTATE if the layer was prefilled.
  */
 int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v,
                       const void* q_last, int P, void* stream);
@@ -103,7 +110,9 @@ int crystalkv_prefill(crystalkv_t* h, int layer, const void* k, const void* v,
  *   q_window   dev [W][batch][Hq][128]   queries of tokens P-W .. P-1
  *   out_window dev [W][batch][Hq][128]   their attention outputs, or NULL
  * All buffers belong to the caller and must stay valid until the work queued on `stream`
- * has run.  1 <= W <= P; P as for crystalkv_prefill.  FullKV mode: only the insertion
+ * has run.  1 <= W <= P, and P <= budget_per_head + max_answer_tokens in evict mode (the window's
+ * outputs need every token's values, so the whole prompt is stored before the one eviction).
+ * FullKV mode: only the insertion
  * (and out_window, if asked for, stays untouched).  Errors: EINVAL; ESTATE if the layer was prefilled.
  */
 int crystalkv_prefill_window(crystalkv_t* h, int layer, const void* k, const void* v,
@@ -264,6 +273,15 @@ int crystalkv_validate(crystalkv_t* h, void* stream);
  * layer is prefilled, ECUDA, ECHECK when ownership is broken.
  */
 int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* stream);
+
+/*
+ * Test hook for the two ownership checks (the paper has no counterpart): overwrites entry
+ * `index` of one head's page table with `page`, both checked against their ranges (EINVAL).
+ * A handle treated this way is inconsistent on purpose: it may be validated and destroyed,
+ * nothing else.  Synchronises `stream`.
+ */
+int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, int32_t index,
+                             int32_t page, void* stream);
 
 const char* crystalkv_strerror(int code);
 const char* crystalkv_last_error(crystalkv_t* h);

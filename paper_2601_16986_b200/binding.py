@@ -34,7 +34,7 @@ class _Cfg(C.Structure):
                 ("budget_per_head", C.c_int32), ("min_budget", C.c_int32), ("max_budget", C.c_int32),
                 ("max_answer_tokens", C.c_int32), ("max_context", C.c_int32), ("top_p", C.c_float),
                 ("lam", C.c_float), ("sm_scale", C.c_float), ("mode", C.c_int32), ("device", C.c_int32),
-                ("evict_every", C.c_int32), ("literal_return", C.c_int32)]
+                ("evict_every", C.c_int32), ("literal_return", C.c_int32), ("budget_ratio", C.c_float)]
 
 
 @dataclass
@@ -57,6 +57,7 @@ class Config:
     dtype: int = BF16
     evict_every: int = 1
     literal_return: int = 0
+    budget_ratio: float = 0.0
 
 
 def declared_symbols():
@@ -98,6 +99,7 @@ def load_library():
     lib.crystalkv_check.argtypes = [vp, vp]
     lib.crystalkv_validate.argtypes = [vp, vp]
     lib.crystalkv_validate_static.argtypes = [vp, vp, vp]
+    lib.crystalkv_debug_set_page.argtypes = [vp, i32, i32, i32, C.c_int32, C.c_int32, vp]
     lib.crystalkv_strerror.argtypes = [i32]
     lib.crystalkv_strerror.restype = C.c_char_p
     lib.crystalkv_last_error.argtypes = [vp]
@@ -129,7 +131,7 @@ class CrystalKV:
         c = _Cfg(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.batch, cfg.dtype,
                  cfg.budget_per_head, cfg.min_budget, cfg.max_budget, cfg.max_answer_tokens,
                  cfg.max_context, cfg.top_p, cfg.lam, cfg.sm_scale, cfg.mode, cfg.device,
-                 cfg.evict_every, cfg.literal_return)
+                 cfg.evict_every, cfg.literal_return, cfg.budget_ratio)
         h = C.c_void_p()
         rc = self.lib.crystalkv_create(C.byref(c), C.byref(h))
         if rc:

@@ -201,7 +201,7 @@ __device__ __forceinline__ void merge_head(const DecodeParams& p, int u, int npi
   }
 }
 
-__global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
+__global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 registers: two LRFU CTAs fit beside it on an SM)
   extern __shared__ __align__(1024) unsigned char smem[];
   const State& st = p.st;
   // Without `early` the kernel before this one may still be writing the lists this one reads.
@@ -246,10 +246,28 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
   auto open_piece = [&](int pi) {
     const int4 dd = __ldg(p.plan.desc + pi);
     const int u = dd.x;
-    f_next = dd.y; f_hi = dd.z;
     f_seq = u / st.H;
     f_ntot = entries_of(u);
-    pt = st.ptab + (size_t)((f_seq * st.L + p.layer) * st.H + (u % st.H)) * st.capg;
+    {   // piece dd.y of dd.z over the head's groups as they are now
+      const unsigned g = (unsigned)(f_ntot + GRP - 1) / GRP;
+      f_next = (int)(g * (unsigned)dd.y / (unsigned)dd.z);
+      f_hi = (int)(g * (unsigned)(dd.y + 1) / (unsigned)dd.z);
+    }
+    const int f_uid = (f_seq * st.L + p.layer) * st.H + (u % st.H);
+    pt = st.ptab + (size_t)f_uid * st.capg;
+    if (p.track) {
+      // The LRFU kernel that follows reads position, tau and CRF of these entries while the next
+      // layer's attention saturates HBM, and every round trip to DRAM costs it microseconds then:
+      // their lines are asked into L2 now (12 bytes per entry against the 512 streamed here).
+      const size_t e0 = (size_t)f_uid * st.cap + (size_t)f_next * GRP, e1 = (size_t)f_uid * st.cap + (size_t)f_hi * GRP;
+      const char* bases[3] = {reinterpret_cast<const char*>(st.meta_pos), reinterpret_cast<const char*>(st.meta_tau),
+                              reinterpret_cast<const char*>(st.meta_crf)};
+      const int nl = (int)(((e1 * 4 + 127) >> 7) - ((e0 * 4) >> 7));   // 128-byte lines per array (arrays are 256-byte aligned)
+      for (int x = lane; x < 3 * nl; x += 32) {
+        const char* a = bases[x / nl] + (((e0 * 4) >> 7) + (x % nl)) * 128;
+        asm volatile("prefetch.global.L2::evict_last [%0];\n" ::"l"(a));
+      }
+    }
     idbase = f_next;
     ids = (f_next + lane < f_hi) ? __ldg(pt + f_next + lane) : 0;   // page ids of groups f_next + lane
     if (lane == 0) fifo[fq_tail & (FIFO - 1)] = pi;
@@ -297,10 +315,12 @@ __global__ void __launch_bounds__(NT, 1) attn_kernel(const DecodeParams p) {
     const int pi = fifo[fq_head & (FIFO - 1)];
     ++fq_head;
     const int4 dd = __ldg(p.plan.desc + pi);
-    const int u = dd.x, lo = dd.y, hi = dd.z, npieces = dd.w >> 16, piece = dd.w & 0xffff;
+    const int u = dd.x, piece = dd.y, npieces = dd.z;
     const int seq = u / st.H;
     const int uid = (seq * st.L + p.layer) * st.H + (u % st.H);
     const int n_tot = entries_of(u);
+    const unsigned g_u = (unsigned)(n_tot + GRP - 1) / GRP;
+    const int lo = (int)(g_u * (unsigned)piece / (unsigned)npieces), hi = (int)(g_u * (unsigned)(piece + 1) / (unsigned)npieces);
     const int hole = p.append ? __ldg(st.hole + uid) : -1;   // where the arriving token goes
     // the G queries as B fragments, running softmax state, O^T accumulators
     uint32_t qb[8][2];

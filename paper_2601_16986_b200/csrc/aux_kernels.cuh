@@ -62,6 +62,142 @@ __global__ void __launch_bounds__(NT) prefill_insert_kernel(State st, int layer,
 }
 
 // ---------------------------------------------------------------------------------------
+// A prompt longer than its heads' budgets is scored before it is stored: Algorithm 1 needs the
+// scores of all P tokens but only the B survivors' rows ever need a place in the pool.
+// Step 1 of three (one CTA per head): the P entries as metadata only (pos = i, CRF 0,
+// tau = P - 1), the scaled logits of the last query's G heads against the prompt's keys, read
+// from the caller's tensors, and the softmax reference point and normaliser per query head, all
+// where the LRFU kernel expects them.
+//   k: [batch][P][H][128]   q_last: [batch][Hq][128]
+__global__ void __launch_bounds__(NT) prefill_score_kernel(State st, Scratch sc, int layer, const __nv_bfloat16* k,
+                                                           const __nv_bfloat16* q_last, int P, int G, float scale,
+                                                           float scale_log2) {
+  __shared__ float s_q[QH * HD];
+  __shared__ float s_red[NW][QH];
+  __shared__ float s_m[QH];
+  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
+  const int uid = (seq * st.L + layer) * st.H + head;
+  const size_t mb = (size_t)uid * st.cap;
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  if (P + 1 > st.cap) {
+    if (tid == 0) { atomicOr(st.errword, ERR_CAPACITY); st.n_cur[uid] = 0; st.hole[uid] = 0; }
+    return;
+  }
+  for (int x = tid; x < QH * HD; x += NT)
+    s_q[x] = (x / HD < G) ? __bfloat162float(q_last[((size_t)u * G + x / HD) * HD + (x % HD)]) : 0.f;
+  __syncthreads();
+  float* S = sc.logits + (size_t)u * sc.cap_s * QH;
+  float mx[QH];
+#pragma unroll
+  for (int g = 0; g < QH; ++g) mx[g] = -INFINITY;
+  for (int i = tid; i < P; i += NT) {
+    st.meta_pos[mb + i] = i;
+    st.meta_tau[mb + i] = P - 1;
+    st.meta_crf[mb + i] = 0.0f;
+    const uint4* row = reinterpret_cast<const uint4*>(k + (((size_t)seq * P + i) * st.H + head) * HD);
+    float acc[QH];
+#pragma unroll
+    for (int g = 0; g < QH; ++g) acc[g] = 0.f;
+    for (int c = 0; c < HD / 8; ++c) {
+      const uint4 v = row[c];
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+      float kv[8];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) { const float2 f = __bfloat1622float2(h2[x]); kv[2 * x] = f.x; kv[2 * x + 1] = f.y; }
+#pragma unroll
+      for (int g = 0; g < QH; ++g)
+#pragma unroll
+        for (int x = 0; x < 8; ++x) acc[g] = fmaf(s_q[g * HD + c * 8 + x], kv[x], acc[g]);
+    }
+    float out[QH];
+#pragma unroll
+    for (int g = 0; g < QH; ++g) {
+      out[g] = __fmul_rn(acc[g], scale);
+      mx[g] = fmaxf(mx[g], acc[g] * scale_log2);
+    }
+    *reinterpret_cast<float4*>(S + (size_t)i * QH) = make_float4(out[0], out[1], out[2], out[3]);
+    *reinterpret_cast<float4*>(S + (size_t)i * QH + 4) = make_float4(out[4], out[5], out[6], out[7]);
+  }
+#pragma unroll
+  for (int g = 0; g < QH; ++g) {
+    const float m = warp_max(mx[g]);
+    if (lane == 0) s_red[w][g] = m;
+  }
+  __syncthreads();
+  if (tid < QH) {
+    float m = s_red[0][tid];
+    for (int x = 1; x < NW; ++x) m = fmaxf(m, s_red[x][tid]);
+    s_m[tid] = m;
+  }
+  __syncthreads();
+  float sum[QH];
+#pragma unroll
+  for (int g = 0; g < QH; ++g) sum[g] = 0.f;
+  const float to_log2 = scale_log2 / scale;
+  for (int i = tid; i < P; i += NT) {
+#pragma unroll
+    for (int g = 0; g < QH; ++g) sum[g] += ex2(S[(size_t)i * QH + g] * to_log2 - s_m[g]);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int g = 0; g < QH; ++g) {
+    const float x = warp_sum(sum[g]);
+    if (lane == 0) s_red[w][g] = x;
+  }
+  __syncthreads();
+  if (tid < G) {
+    float l = 0.f;
+    for (int x = 0; x < NW; ++x) l += s_red[x][tid];
+    sc.mfin[u * (2 * QH) + tid] = s_m[tid];
+    sc.mfin[u * (2 * QH) + QH + tid] = l;
+  }
+  if (tid == 0) { st.n_cur[uid] = P; st.hole[uid] = P; st.npages[uid] = 0; }
+}
+
+// Step 3 (step 2 is the LRFU kernel, which leaves the survivors' metadata dense): the pages that
+// back the survivors and the place of the next arrival are taken from the free list and the
+// survivors' rows are fetched from the prompt tensors by their token positions.
+__global__ void __launch_bounds__(NT) prefill_rows_kernel(State st, int layer, const __nv_bfloat16* k,
+                                                          const __nv_bfloat16* v, int P) {
+  __shared__ int s_top;
+  const int u = blockIdx.x, seq = u / st.H, head = u % st.H;
+  const int uid = (seq * st.L + layer) * st.H + head;
+  const size_t mb = (size_t)uid * st.cap;
+  const int tid = threadIdx.x;
+  const int n = st.n_cur[uid];
+  const int need = n / GRP + 1;
+  if (tid == 0) {
+    int top = atomicSub(&st.free_top[seq], need);
+    if (top < need) {
+      atomicAdd(&st.free_top[seq], need);
+      atomicOr(st.errword, ERR_FREE_UNDERFLOW);
+      top = -1;
+    }
+    s_top = top;
+  }
+  __syncthreads();
+  const int top = s_top;
+  if (top < 0) {
+    if (tid == 0) { st.n_cur[uid] = 0; st.hole[uid] = 0; }
+    return;
+  }
+  const int* stack = st.free_stack + (size_t)seq * st.pages_per_seq;
+  int* pt = st.ptab + (size_t)uid * st.capg;
+  for (int j = tid; j < need; j += NT) pt[j] = stack[top - 1 - j];
+  unsigned char* poolseq = st.pool + (size_t)seq * st.pages_per_seq * PAGE_BYTES;
+  const int c = tid & 31;
+  for (int i = tid >> 5; i < n; i += NW) {
+    const int page = stack[top - 1 - (i >> 4)];
+    const int tok = min(max(st.meta_pos[mb + i], 0), P - 1);
+    const size_t off = (((size_t)seq * P + tok) * st.H + head) * HD * 2;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(c < 16 ? k : v) + off + (c & 15) * 16;
+    *reinterpret_cast<uint4*>(poolseq + (size_t)page * PAGE_BYTES + chunk_offset(i & (GRP - 1), c)) =
+        *reinterpret_cast<const uint4*>(src);
+  }
+  if (tid == 0) st.npages[uid] = need;
+}
+
+// ---------------------------------------------------------------------------------------
 // Brings one step's q, k_new and v_new from page-locked host memory (read over the bus through
 // its device mapping, 16 bytes per thread) into the staging buffers: one launch instead of three
 // copies.  It runs in the caller's stream directly ahead of the step's attention kernel, both

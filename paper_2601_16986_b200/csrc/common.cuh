@@ -58,13 +58,16 @@ struct State {
   int batch, L, H, cap, capg;
 };
 
-// Launch plan of one layer, written by the kernel that last changed the layer's lengths and read
-// by the next attention launch: all groups of the layer's heads laid in a row and cut into
-// nearly equal runs, one run per streaming warp; a run is one piece per head it overlaps.
+// Launch plan of one layer, read by its next attention launch: every head cut into k pieces of
+// nearly equal length, one piece per streaming warp (plan.cuh).  A piece is named by (head, j, k)
+// and covers groups [g j / k, g (j + 1) / k) of the head's g groups AT LAUNCH TIME, so a plan stays
+// correct when heads grow or shrink by a few entries; it is rewritten when a head's group count has
+// drifted from the one it was made for by an eighth (at least two), and after every reallocation.
 struct Plan {
-  int4* desc;        // [pd_cap] pieces in row order: {head index u, first group, end group, (pieces of u << 16) | piece index}
+  int4* desc;        // [pd_cap] pieces, head after head: {head index u, piece j, pieces k of the head, 0}
   int2* wrange;      // [warps] pieces [x, y) of the physical warp cta * NW + w
   int* npc;          // [U] pieces per head
+  int* gplan;        // [U] groups per head the plan was made for
   int* hdr;          // [4] pieces in total, groups in total, warps the plan was made for, append it was made for
 };
 
@@ -87,7 +90,8 @@ struct DecodeParams {
   const __nv_bfloat16* k_new;   // [batch][H][128]
   const __nv_bfloat16* v_new;
   __nv_bfloat16* out;           // [batch][Hq][128]
-  int* done_ctr;     // LRFU kernel: counts its finished CTAs; the last one writes the layer's next plan
+  int* done_ctr;     // LRFU kernel: [0] counts its finished CTAs, [1] set when a head's group count changed: the
+                     // last CTA then writes the layer's next plan
   int layer;
   int G;          // query heads per kv head
   int t;          // time of this step
@@ -100,6 +104,8 @@ struct DecodeParams {
   int hold;       // 1: Algorithm 1 stops after step 3; lengths and lists stay as they are
   int evict_every;   // m >= 1: step 4 waits until a head is m entries over its budget, then removes them all
   int literal;    // 1: Algorithm 1 is skipped for a head below its budget (its first line as printed)
+  int rows_absent;   // 1: the heads' entries are only metadata so far (a prompt being scored before its
+                     //    survivors' rows are stored): nothing touches pool pages
   int plan_append;   // what the plan the LRFU kernel leaves behind is for: 1 = a decode step, 0 = a scoring pass
   int plan_warps;    // warps of the attention grid the plan is made for
   int plan_grid;     // CTAs of that grid

@@ -44,15 +44,17 @@ struct crystalkv {
   float* sc_mfin[NSETS] = {};
   float* sc_partials[2] = {};
   int* sc_ticket[2] = {};
-  float* sc_pbar = nullptr;
+  float* sc_pbar[2] = {};          // one per internal stream
   int* piece_ctr = nullptr;
   int cap_s = 0, pmax = 0;
   long long nA = 0;                // attention launches so far
   std::vector<int> t_layer;        // per layer: time of the last step
   // LRFU launches are numbered; launch k uses scratch set k % NSETS and event k % EV_RING
   static constexpr int EV_RING = 32;
-  cudaStream_t side = nullptr;
-  cudaEvent_t evA = nullptr, evF[EV_RING] = {};
+  // two internal streams taken in turn: the LRFU kernels of consecutive layers do not depend on
+  // one another, so the second may fill SM room as the first one's CTAs finish
+  cudaStream_t side[2] = {};
+  cudaEvent_t evA[EV_RING] = {}, evF[EV_RING] = {};
   long long kF = 0, joined = -1;
   std::vector<long long> lastF;    // per layer: number of its latest LRFU launch, -1 = none
   int prev_layer = -1;             // layer of the launch pair issued last, -1 after any other call
@@ -208,7 +210,23 @@ int validate(const crystalkv_config_t* c, std::string& why) {
   if (c->device < 0 || c->device >= MAX_DEVICES) { why = "device ordinal outside [0, 64)"; return CRYSTALKV_EINVAL; }
   if (c->evict_every < 0 || c->evict_every > 4096) { why = "evict_every outside [0, 4096]"; return CRYSTALKV_EINVAL; }
   if (c->literal_return != 0 && c->literal_return != 1) { why = "literal_return must be 0 or 1"; return CRYSTALKV_EINVAL; }
+  if (!(c->budget_ratio >= 0.f) || c->budget_ratio > 1.f) { why = "budget_ratio outside [0, 1]"; return CRYSTALKV_EINVAL; }
   return CRYSTALKV_OK;
+}
+
+// Ratio budgets: the average budget per head after `tokens` tokens, floor(r * tokens) in fp64 from
+// the fp32 ratio, kept within [max(1, min_budget), budget_per_head].
+int ratio_budget(const crystalkv_config_t& c, int tokens) {
+  long long b = (long long)std::floor((double)c.budget_ratio * (double)tokens);
+  b = std::max<long long>(b, std::max(1, c.min_budget));
+  b = std::min<long long>(b, c.budget_per_head);
+  return (int)b;
+}
+
+// Sets the budget of every head of one layer.
+__global__ void fill_layer_budget_kernel(State st, int layer, int v) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u < st.batch * st.H) st.budget[((u / st.H) * st.L + layer) * st.H + (u % st.H)] = v;
 }
 
 int check_layer(crystalkv_t* h, int layer) {
@@ -230,10 +248,10 @@ DecodeParams make_params(crystalkv_t* h, int layer) {
   DecodeParams p{};
   p.st = h->st;
   p.plan = h->plans[layer];
-  p.done_ctr = h->done_ctr;
+  p.done_ctr = h->done_ctr;   // (launch_step picks the internal stream's own)
   p.sc.cap_s = h->cap_s;
   p.sc.pmax = h->pmax;
-  p.sc.pbar = h->sc_pbar;
+  p.sc.pbar = h->sc_pbar[0];
   p.sc.partials = h->sc_partials[h->nA & 1];
   p.sc.ticket = h->sc_ticket[h->nA & 1];
   p.sc.logits = h->sc_logits[0];
@@ -263,6 +281,7 @@ int replan(crystalkv_t* h, int layer0, int count, int append, int n_limit, cudaS
 int join_side(crystalkv_t* h, cudaStream_t s) {
   h->prev_layer = -1;
   if (h->kF > 0) CK(h, cudaStreamWaitEvent(s, h->evF[(h->kF - 1) % crystalkv::EV_RING], 0));
+  if (h->kF > 1) CK(h, cudaStreamWaitEvent(s, h->evF[(h->kF - 2) % crystalkv::EV_RING], 0));   // the other internal stream
   h->joined = h->kF - 1;
   if (h->nHost > 0) CK(h, cudaStreamWaitEvent(s, h->evOut[(h->nHost - 1) % crystalkv::HOST_RING], 0));   // copies back run in order
   return CRYSTALKV_OK;
@@ -275,7 +294,8 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
   const long long k = h->kF;
   if (track) {
     // launch k reuses the scratch of launch k - NSETS and continues the state its layer's
-    // previous LRFU launch wrote; the internal stream runs in order, so one event covers both
+    // previous LRFU launch wrote; each internal stream runs in order, so the events of two
+    // consecutive launches cover everything before them
     // A wait on the caller's stream costs several microseconds (the attention kernel behind it
     // no longer starts early), so one wait covers as many launches as the sets allow: it targets
     // the newest LRFU launch that has had two attention kernels' time to finish.
@@ -283,6 +303,7 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
     if (need >= 0 && need > h->joined) {
       const long long target = std::max(need, k - 3);
       CK(h, cudaStreamWaitEvent(s, h->evF[target % crystalkv::EV_RING], 0));
+      if (target > 0) CK(h, cudaStreamWaitEvent(s, h->evF[(target - 1) % crystalkv::EV_RING], 0));   // the other internal stream
       h->joined = target;
     }
     p.sc.logits = h->sc_logits[k % NSETS];
@@ -308,10 +329,14 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
   }
   h->prev_layer = layer;
   if (track) {
-    CK(h, cudaEventRecord(h->evA, s));
-    CK(h, cudaStreamWaitEvent(h->side, h->evA, 0));
-    CK(h, lrfu_dispatch(h->G, p, h->U, h->side));
-    CK(h, cudaEventRecord(h->evF[k % crystalkv::EV_RING], h->side));
+    const int si = (int)(k & 1);
+    cudaEvent_t ea = h->evA[k % crystalkv::EV_RING];
+    p.sc.pbar = h->sc_pbar[si];
+    p.done_ctr = h->done_ctr + 2 * si;
+    CK(h, cudaEventRecord(ea, s));
+    CK(h, cudaStreamWaitEvent(h->side[si], ea, 0));
+    CK(h, lrfu_dispatch(h->G, p, h->U, h->side[si]));
+    CK(h, cudaEventRecord(h->evF[k % crystalkv::EV_RING], h->side[si]));
     h->lastF[layer] = k;
     h->kF = k + 1;
   }
@@ -340,7 +365,8 @@ int crystalkv_destroy(crystalkv_t* h) {
   if (!h) return CRYSTALKV_OK;
   DeviceScope scope(h->cfg.device);
   cudaDeviceSynchronize();
-  if (h->side) cudaStreamDestroy(h->side);
+  for (cudaStream_t x : h->side)
+    if (x) cudaStreamDestroy(x);
   if (h->copy_in) cudaStreamDestroy(h->copy_in);
   if (h->copy_out) cudaStreamDestroy(h->copy_out);
   for (int i = 0; i < crystalkv::HOST_RING; ++i) {
@@ -348,7 +374,8 @@ int crystalkv_destroy(crystalkv_t* h) {
     if (h->evUse[i]) cudaEventDestroy(h->evUse[i]);
     if (h->evOut[i]) cudaEventDestroy(h->evOut[i]);
   }
-  if (h->evA) cudaEventDestroy(h->evA);
+  for (cudaEvent_t e : h->evA)
+    if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : h->evF)
     if (e) cudaEventDestroy(e);
   for (void* p : h->allocs) cudaFree(p);
@@ -421,10 +448,13 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   h->smem = RING_BYTES + NW * STAGES * 8 + NW * FIFO * sizeof(int);
   int bps = 0;
   CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem));
+  // The largest shared-memory carve-out, although the ring alone would fit a smaller one: the CTAs
+  // of the LRFU kernel have to find room beside an attention CTA on the same SM.
+  CKC(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
   CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
   if (bps < 1) { h->err = "attention kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
   h->grid = h->num_sms * bps;
-  CKC(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
+  for (cudaStream_t& x : h->side) CKC(cudaStreamCreateWithFlags(&x, cudaStreamNonBlocking));
   CKC(cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking));
   CKC(cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking));
   for (int i = 0; i < crystalkv::HOST_RING; ++i) {
@@ -432,7 +462,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     CKC(cudaEventCreateWithFlags(&h->evUse[i], cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&h->evOut[i], cudaEventDisableTiming));
   }
-  CKC(cudaEventCreateWithFlags(&h->evA, cudaEventDisableTiming));
+  for (cudaEvent_t& e : h->evA) CKC(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
   for (cudaEvent_t& e : h->evF) CKC(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
 
   State& st = h->st;
@@ -452,19 +482,21 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   // launch plans, one per layer: at most one piece per warp and one more per head
   {
     const int nWarps = h->grid * NW, pd_cap = nWarps + h->U;
-    int4* desc = nullptr; int2* wr = nullptr; int *npc = nullptr, *hdr = nullptr;
+    int4* desc = nullptr; int2* wr = nullptr; int *npc = nullptr, *gpl = nullptr, *hdr = nullptr;
     DA(&desc, (size_t)c.n_layers * pd_cap);
     DA(&wr, (size_t)c.n_layers * nWarps);
     DA(&npc, (size_t)c.n_layers * h->U);
+    DA(&gpl, (size_t)c.n_layers * h->U);
     DA(&hdr, (size_t)c.n_layers * 4);
     CKC(cudaMemset(hdr, 0, (size_t)c.n_layers * 4 * sizeof(int)));
     h->plans.resize(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l)
-      h->plans[l] = Plan{desc + (size_t)l * pd_cap, wr + (size_t)l * nWarps, npc + (size_t)l * h->U, hdr + (size_t)l * 4};
+      h->plans[l] = Plan{desc + (size_t)l * pd_cap, wr + (size_t)l * nWarps, npc + (size_t)l * h->U, gpl + (size_t)l * h->U,
+                         hdr + (size_t)l * 4};
     DA(&h->d_plans, c.n_layers);
     CKC(cudaMemcpy(h->d_plans, h->plans.data(), (size_t)c.n_layers * sizeof(Plan), cudaMemcpyHostToDevice));
-    DA(&h->done_ctr, 1);
-    CKC(cudaMemset(h->done_ctr, 0, sizeof(int)));
+    DA(&h->done_ctr, 4);   // per internal stream: finished CTAs of its running LRFU kernel; whether the layer's plan went stale
+    CKC(cudaMemset(h->done_ctr, 0, 4 * sizeof(int)));
   }
   DA(&h->tab, (size_t)c.max_context + 1);
   st.tab = h->tab;
@@ -483,7 +515,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
     DA(&h->sc_ticket[i], h->U);
     CKC(cudaMemset(h->sc_ticket[i], 0, (size_t)h->U * sizeof(int)));
   }
-  DA(&h->sc_pbar, (size_t)h->U * h->cap_s);
+  for (int i = 0; i < 2; ++i) DA(&h->sc_pbar[i], (size_t)h->U * h->cap_s);
   DA(&h->piece_ctr, 4);
   CKC(cudaMemset(h->piece_ctr, 0, 4 * sizeof(int)));
   const size_t qn = (size_t)c.batch * c.n_q_heads * HD, kn = (size_t)c.batch * c.n_kv_heads * HD;
@@ -523,7 +555,8 @@ int crystalkv_set_stage(crystalkv_t* h, int stage) {
   if (stage == CRYSTALKV_STAGE_THINK && h->answer_steps > 0)
     return fail(h, CRYSTALKV_ESTATE, "answer tokens were appended; the think stage cannot resume");
   ON_DEVICE(h);
-  if (stage != h->stage) CK(h, cudaStreamSynchronize(h->side));   // no LRFU kernel is left behind the switch
+  if (stage != h->stage)   // no LRFU kernel is left behind the switch
+    for (cudaStream_t x : h->side) CK(h, cudaStreamSynchronize(x));
   h->prev_layer = -1;
   h->stage = stage;
   return CRYSTALKV_OK;
@@ -544,14 +577,41 @@ static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* 
   const crystalkv_config_t& c = h->cfg;
   const bool evict = c.mode == CRYSTALKV_MODE_EVICT;
   if (P < 1) return fail(h, CRYSTALKV_EINVAL, "P must be >= 1");
-  if (evict && P > c.budget_per_head + c.max_answer_tokens)
-    return fail(h, CRYSTALKV_EINVAL, "prompt longer than budget_per_head + max_answer_tokens");
+  // A prompt beyond the budget is scored from the caller's tensors and only its survivors are
+  // stored; with an observation window the whole prompt must fit the pool for a moment (the
+  // window's attention outputs need the values).
+  const bool score_first = evict && W == 0 && P > (c.budget_ratio > 0.f ? ratio_budget(c, P) : c.budget_per_head);
+  if (evict && !score_first && P > c.budget_per_head + c.max_answer_tokens)
+    return fail(h, CRYSTALKV_EINVAL, "prompt with an observation window longer than budget_per_head + max_answer_tokens");
+  if (evict && P + 1 > h->cap) return fail(h, CRYSTALKV_EINVAL, "prompt longer than the heads' list capacity (max_budget + evict_every + max_answer_tokens)");
   if (P >= c.max_context) return fail(h, CRYSTALKV_EINVAL, "prompt reaches max_context");
   if (h->t_layer[layer] >= 0) return fail(h, CRYSTALKV_ESTATE, "layer already prefilled");
   ON_DEVICE(h);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   rc = join_side(h, s);   // the insertion takes pages; no LRFU kernel may take or return any meanwhile
   if (rc) return rc;
+  if (evict && c.budget_ratio > 0.f) {   // the prompt's share of the context
+    fill_layer_budget_kernel<<<(h->U + NT - 1) / NT, NT, 0, s>>>(h->st, layer, ratio_budget(c, P));
+    CK(h, cudaGetLastError());
+  }
+  if (score_first) {
+    // Algorithm 1 with the last query over metadata and logits only; every kernel on `s`, which has
+    // joined the internal stream, so any scratch set is free
+    DecodeParams p = make_params(h, layer);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.t = P - 1;
+    p.append = 0; p.track = 1; p.release = 1; p.rows_absent = 1; p.plan_append = 1;
+    prefill_score_kernel<<<h->U, NT, 0, s>>>(h->st, p.sc, layer, static_cast<const __nv_bfloat16*>(k), p.q, P, h->G,
+                                             p.scale, p.scale_log2);
+    CK(h, cudaGetLastError());
+    CK(h, lrfu_dispatch(h->G, p, h->U, s));
+    prefill_rows_kernel<<<h->U, NT, 0, s>>>(h->st, layer, static_cast<const __nv_bfloat16*>(k),
+                                            static_cast<const __nv_bfloat16*>(v), P);
+    CK(h, cudaGetLastError());
+    h->prev_layer = -1;
+    h->t_layer[layer] = P - 1;
+    return CRYSTALKV_OK;
+  }
   prefill_insert_kernel<<<h->U, NT, 0, s>>>(h->st, layer, static_cast<const __nv_bfloat16*>(k),
                                             static_cast<const __nv_bfloat16*>(v), P, W > 0 ? 1 : 0);
   CK(h, cudaGetLastError());
@@ -717,11 +777,11 @@ int crystalkv_rebudget(crystalkv_t* h, void* stream) {
   const int N = c.n_layers * c.n_kv_heads;
   const size_t sm = (size_t)N * (3 * sizeof(double) + sizeof(long long) + 2 * sizeof(int)) + (size_t)c.n_layers * 2 * sizeof(double);
   if (sm > 48 * 1024) CK(h, cudaFuncSetAttribute(alg2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
-  const long long B_total = (long long)c.budget_per_head * N;
+  const long long B_total = (long long)(c.budget_ratio > 0.f ? ratio_budget(c, t_last + 1) : c.budget_per_head) * N;
   alg2_kernel<<<c.batch, NT, sm, s>>>(h->Asum, h->st.budget, c.n_layers, c.n_kv_heads, B_total, c.min_budget, c.max_budget);
   CK(h, cudaGetLastError());
   for (int l = 0; l < c.n_layers; ++l) {
-    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, l, t_last, reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, l, t_last, reinterpret_cast<int*>(h->sc_pbar[0]), h->cap_s);
     CK(h, cudaGetLastError());
   }
   // heads changed length: every layer's next decode step needs a new plan
@@ -741,7 +801,7 @@ int crystalkv_set_budget(crystalkv_t* h, int layer, int seq, int kv_head, int32_
   CK(h, cudaMemcpyAsync(h->st.budget + uid, &budget, sizeof(int), cudaMemcpyHostToDevice, s));
   CK(h, cudaStreamSynchronize(s));
   if (h->t_layer[layer] >= 0) {
-    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, layer, h->t_layer[layer], reinterpret_cast<int*>(h->sc_pbar), h->cap_s);
+    shrink_kernel<<<h->U, NT, 0, s>>>(h->st, layer, h->t_layer[layer], reinterpret_cast<int*>(h->sc_pbar[0]), h->cap_s);
     CK(h, cudaGetLastError());
     return replan(h, layer, 1, 1, 0, s);
   }
@@ -974,6 +1034,20 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
   if (res[0] || res[1])
     return fail(h, CRYSTALKV_ECHECK, "page ownership broken: " + std::to_string(res[0]) + " ids or counts out of range, " +
                                          std::to_string(res[1]) + " pages not owned exactly once");
+  return CRYSTALKV_OK;
+}
+
+int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, int32_t index, int32_t page, void* stream) {
+  int rc = check_unit(h, layer, seq, kv_head);
+  if (rc) return rc;
+  if (index < 0 || index >= h->st.capg || page < 0 || page >= h->pages_per_seq)
+    return fail(h, CRYSTALKV_EINVAL, "page table index or page id out of range");
+  ON_DEVICE(h);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
+  const int uid = (seq * h->cfg.n_layers + layer) * h->cfg.n_kv_heads + kv_head;
+  CK(h, cudaMemcpyAsync(h->st.ptab + (size_t)uid * h->st.capg + index, &page, sizeof(int), cudaMemcpyHostToDevice, s));
+  CK(h, cudaStreamSynchronize(s));
   return CRYSTALKV_OK;
 }
 

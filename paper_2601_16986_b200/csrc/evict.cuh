@@ -32,9 +32,12 @@ __device__ __forceinline__ bool key_le(const Key96& a, const uint32_t* b) {
 
 // Moves the entry at list position `src` of a head to position `dst` (one warp: lane c carries
 // chunk c of the 512-byte row, which sits at a different place in the two pages' layouts).
-__device__ __forceinline__ void move_entry(const State& st, int uid, int seq, size_t mb, int dst, int src, int lane) {
-  const uint4 v = *reinterpret_cast<const uint4*>(entry_chunk(st, uid, seq, src, lane));
-  *reinterpret_cast<uint4*>(entry_chunk(st, uid, seq, dst, lane)) = v;
+__device__ __forceinline__ void move_entry(const State& st, int uid, int seq, size_t mb, int dst, int src, int lane,
+                                           bool rows = true) {
+  if (rows) {
+    const uint4 v = *reinterpret_cast<const uint4*>(entry_chunk(st, uid, seq, src, lane));
+    *reinterpret_cast<uint4*>(entry_chunk(st, uid, seq, dst, lane)) = v;
+  }
   if (lane == 0) {
     st.meta_pos[mb + dst] = st.meta_pos[mb + src];
     st.meta_tau[mb + dst] = st.meta_tau[mb + src];
@@ -60,8 +63,10 @@ __device__ __forceinline__ void release_pages(const State& st, int uid, int seq,
 
 // Removes the k lowest entries (1 <= k < n) of head `uid` at time t; the head's n entries must be
 // dense (list positions 0 .. n-1).  `sh` is >= 1.2 KB (300 ints) of shared scratch, `tmp` a global
-// int scratch of >= n words.  All NT threads call it.
-__device__ void evict_many(const State& st, int uid, int seq, int n, int k, int t, bool release, int* sh, int* tmp) {
+// int scratch of >= n words.  rows = false: the entries have no rows in the pool yet (a prompt
+// that is being scored), only their metadata moves.  All NT threads call it.
+__device__ void evict_many(const State& st, int uid, int seq, int n, int k, int t, bool release, int* sh, int* tmp,
+                           bool rows = true) {
   const size_t mb = (size_t)uid * st.cap;
   int* hist = sh;             // 256
   int* s_kw = sh + 256;       // 3 words of the k-th key
@@ -147,14 +152,14 @@ __device__ void evict_many(const State& st, int uid, int seq, int n, int k, int 
   }
   __syncthreads();
   // every mover fills one gap, in order; rows and metadata travel together
-  for (int j = tid >> 5; j < min(gaps, movers); j += NW) move_entry(st, uid, seq, mb, tmp[j], tmp[gaps + j], tid & 31);
+  for (int j = tid >> 5; j < min(gaps, movers); j += NW) move_entry(st, uid, seq, mb, tmp[j], tmp[gaps + j], tid & 31, rows);
   __syncthreads();
   if (tid == 0) {
     st.n_cur[uid] = nk;
     st.hole[uid] = nk;
     atomicAdd(&st.counters[2], (unsigned long long)k);
   }
-  if (release) release_pages(st, uid, seq, nk, s_krem);
+  if (release && rows) release_pages(st, uid, seq, nk, s_krem);
 }
 
 }  // namespace ckv

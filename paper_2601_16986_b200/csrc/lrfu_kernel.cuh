@@ -81,7 +81,7 @@ __device__ __forceinline__ unsigned long long mass_of(float pm) { return (unsign
 // EPT > 0: every thread keeps the pbar of its entries tid, tid + NT, ... (at most EPT) in
 // registers; EPT == 0: they live in the global scratch and any n is allowed.
 template <int G, int EPT>
-__device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n, LrfuSmem& sh, const Front<G>& fr) {
+__device__ int lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n, LrfuSmem& sh, const Front<G>& fr) {
   constexpr int R = EPT > 0 ? EPT : 1;
   const State& st = p.st;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -146,23 +146,33 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       }
     }
   } else if (EPT > 0) {
-    // batches of four entries: their rows are requested together (clamped index, no branch)
+    // batches of BR entries whose rows are requested together (clamped index, no branch): while the
+    // attention kernel saturates HBM every dependent round of loads costs this CTA microseconds, so
+    // a batch is as large as the registers allow (only the G logits of a row are loaded)
+    constexpr int BR = G <= 5 ? 8 : 4;
 #pragma unroll
     for (int k = 0; k < R; ++k) pmr[k] = 0.f;
 #pragma unroll
-    for (int k0 = 0; k0 < R; k0 += 4) {
+    for (int k0 = 0; k0 < R; k0 += BR) {
       if (k0 < kmax) {
-        float4 ra[4], rb[4];
+        float4 ra[BR];
+        float rb[BR][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < BR; ++j) {
           const int i = min(tid + (k0 + j) * NT, n - 1);
           ra[j] = ld_f32x4(S + (size_t)i * QH);
-          rb[j] = (G > 4) ? ld_f32x4(S + (size_t)i * QH + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          if (G == 5) {
+            rb[j][0] = ld_f32(S + (size_t)i * QH + 4);
+          } else if (G > 5) {
+            const float4 t4 = ld_f32x4(S + (size_t)i * QH + 4);
+            rb[j][0] = t4.x; rb[j][1] = t4.y; rb[j][2] = t4.z; rb[j][3] = t4.w;
+          }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < BR; ++j) {
           if (k0 + j < R) {
-            const float sv[8] = {ra[j].x, ra[j].y, ra[j].z, ra[j].w, rb[j].x, rb[j].y, rb[j].z, rb[j].w};
+            const float sv[8] = {ra[j].x, ra[j].y, ra[j].z, ra[j].w, G > 4 ? rb[j][0] : 0.f, G > 5 ? rb[j][1] : 0.f,
+                                 G > 6 ? rb[j][2] : 0.f, G > 7 ? rb[j][3] : 0.f};
             float pm = 0.f;
 #pragma unroll
             for (int g = 0; g < G; ++g) pm = fmaf(expf(sv[g] - mx[g]), invl[g], pm);
@@ -410,23 +420,23 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
       if (less) { bk0 = c0; bk1 = c1; bk2 = c2; bidx = i; }
     }
   };
-  if (EPT > 8) {   // many entries per thread: four at a time, their stored state requested together
+  if (EPT > 8) {   // many entries per thread: eight at a time, their stored state requested together
 #pragma unroll
-    for (int k0 = 0; k0 < R; k0 += 4) {
+    for (int k0 = 0; k0 < R; k0 += 8) {
       if (k0 < kmax) {
-        int pos4[4], tau4[4];
-        float crf4[4], dec4[4];
+        int pos4[8], tau4[8];
+        float crf4[8], dec4[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 8; ++j) {
           const size_t i = mb + min(tid + (k0 + j) * NT, n - 1);
           pos4[j] = ld_i32(st.meta_pos + i);
           tau4[j] = ld_i32(st.meta_tau + i);
           crf4[j] = ld_f32(st.meta_crf + i);
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) dec4[j] = __ldg(st.tab + (p.t - min(tau4[j], p.t)));
+        for (int j = 0; j < 8; ++j) dec4[j] = __ldg(st.tab + (p.t - min(tau4[j], p.t)));
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 8; ++j) {
           const int i = tid + (k0 + j) * NT;
           if (k0 + j < R && i < n) update(i, pmr[k0 + j < R ? k0 + j : 0], pos4[j], tau4[j], crf4[j], dec4[j]);
         }
@@ -479,10 +489,12 @@ __device__ void lrfu_unit(const DecodeParams& p, int u, int uid, int seq, int n,
   } else if (k_evict > 1) {
     __syncthreads();
     if (p.append && k_evict > p.evict_every && tid == 0) atomicOr(st.errword, ERR_OVER_EVICT);
-    evict_many(st, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh.ev, reinterpret_cast<int*>(pbar));
+    evict_many(st, uid, seq, n, min(k_evict, n - 1), p.t, p.release != 0, sh.ev, reinterpret_cast<int*>(pbar),
+               p.rows_absent == 0);
     n_after = n - min(k_evict, n - 1);
   }
   if (n_after == n && tid == 0 && !p.hold) keep_all(st, uid, seq, n, p.append != 0);
+  return n_after;   // the head's length after the step
 }
 
 template <int G>
@@ -494,8 +506,10 @@ __global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
   // one batch of requests: the length, the budget, the softmax reference, and the logit rows the
   // common path needs (requested for a full thread's worth, clamped to the scratch)
   int n_raw = ld_i32(st.n_cur + uid);
+  const int g_plan = (threadIdx.x == 0 && p.plan_append >= 0) ? ld_i32(p.plan.gplan + u) : 0;   // used at the very end
   if (p.n_limit > 0) n_raw = min(n_raw, p.n_limit);
   const int n = n_raw + p.append;
+  int n_new = n;   // the head's length after this launch
   if (p.track) {
     Front<G> fr;
     fr.budget = ld_i32(st.budget + uid);
@@ -515,27 +529,40 @@ __global__ void __launch_bounds__(NT, 5) lrfu_kernel(const DecodeParams p) {
     }
     if (n <= 0) {
       if (threadIdx.x == 0 && !p.hold) { st.n_cur[uid] = 0; st.hole[uid] = 0; }
+      n_new = 0;
     } else if (p.literal && n < fr.budget) {   // Algorithm 1's first line as printed: nothing runs below the budget
       if (threadIdx.x == 0 && !p.hold) keep_all(st, uid, seq, n, p.append != 0);
     } else if (n <= FRONT * NT) {
-      lrfu_unit<G, FRONT>(p, u, uid, seq, n, sh, fr);
+      n_new = lrfu_unit<G, FRONT>(p, u, uid, seq, n, sh, fr);
+    } else if (n <= 10 * NT) {
+      n_new = lrfu_unit<G, 10>(p, u, uid, seq, n, sh, fr);
     } else if (n <= 17 * NT) {
-      lrfu_unit<G, 17>(p, u, uid, seq, n, sh, fr);
+      n_new = lrfu_unit<G, 17>(p, u, uid, seq, n, sh, fr);
     } else {
-      lrfu_unit<G, 0>(p, u, uid, seq, n, sh, fr);
+      n_new = lrfu_unit<G, 0>(p, u, uid, seq, n, sh, fr);
     }
   } else if (threadIdx.x == 0) {
     keep_all(st, uid, seq, n, p.append != 0);   // no Algorithm 1: the head keeps its new entry
   }
   if (threadIdx.x == 0) atomicAdd(&st.counters[0], (unsigned long long)max(n, 0));
   if (p.plan_append < 0) return;
-  // ---- the CTA that finishes last knows every head's new length: it writes the layer's next plan
-  __syncthreads();
+  // ---- The layer's plan names pieces by (head, j of k), so it stays correct while heads grow or
+  // shrink a little; a head whose group count has drifted from the planned one by an eighth (at
+  // least two), or a next launch of another kind than this one, marks it stale, and the CTA that
+  // finishes last (it then knows every head's new length) writes a new one.  In steady state (one
+  // entry arrives, one leaves) nothing is written.  Thread 0 wrote the head's new length itself,
+  // so the release of its count makes that length visible to whoever acquires the last count.
   if (threadIdx.x == 0) {
-    __threadfence();
-    const int done = atomicAdd(p.done_ctr, 1);
-    sh.is_last = (done == (int)gridDim.x - 1);
-    if (sh.is_last) { *p.done_ctr = 0; __threadfence(); }
+    const int g_new = (n_new + p.plan_append + GRP - 1) / GRP;
+    if (abs(g_new - g_plan) >= max(2, g_plan >> 3) || p.append != p.plan_append) atomicOr(p.done_ctr + 1, 1);
+    int done;
+    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(done) : "l"(p.done_ctr) : "memory");
+    int last = (done == (int)gridDim.x - 1);
+    if (last) {
+      *p.done_ctr = 0;
+      last = atomicExch(p.done_ctr + 1, 0);   // stale?
+    }
+    sh.is_last = last;
   }
   __syncthreads();
   if (!sh.is_last) return;

@@ -7,9 +7,10 @@
 // round the SMs one by one, so every SM streams the same number of them to within one.  With
 // more heads than warps every head is one piece and a warp takes several in turn.  A head of
 // several pieces is merged from their partial results.  The plan only depends on the heads'
-// lengths, so it is written by whichever kernel changed them last (the LRFU kernel of the layer's
-// previous step, the shrink pass of a reallocation, the prompt insertion) and the attention
-// kernel starts streaming without deriving anything.
+// lengths, so it is written by whichever kernel changed them (the LRFU kernel of the layer's
+// previous step once a head has drifted from the planned length, the shrink pass of a
+// reallocation, the prompt insertion) and the attention kernel starts streaming without deriving
+// anything but its pieces' bounds from the heads' current lengths.
 #pragma once
 #include "common.cuh"
 
@@ -18,7 +19,7 @@ namespace ckv {
 // Called by all NT threads of one CTA.  `gs` is shared memory for U + 1 ints, `red` for NW + 1.
 // append: the plan is for a decode step (every head one entry longer than now); n_limit > 0: for
 // a scoring pass over the first n_limit entries of every head.
-__device__ __noinline__ void write_plan(const State& st, const Plan& pl, int layer, int append, int n_limit, int nWarps,
+__device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int layer, int append, int n_limit, int nWarps,
                                         int grid, int* gs, int* red) {
   const int U = st.batch * st.H, tid = threadIdx.x;
   // ---- groups per head
@@ -73,9 +74,8 @@ __device__ __noinline__ void write_plan(const State& st, const Plan& pl, int lay
     pieces += tot;
     if (u < U) {
       pl.npc[u] = k;
-      for (int j = 0; j < k; ++j)
-        pl.desc[start + j] = make_int4(u, (int)((unsigned)g * (unsigned)j / (unsigned)k),
-                                       (int)((unsigned)g * (unsigned)(j + 1) / (unsigned)k), (k << 16) | j);
+      pl.gplan[u] = g;
+      for (int j = 0; j < k; ++j) pl.desc[start + j] = make_int4(u, j, k, 0);
     }
   }
   // ---- which warp takes which pieces: piece i goes to CTA i % grid, warp i / grid; with more

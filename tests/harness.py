@@ -44,25 +44,26 @@ class Report:
 
 class LockStep:
     def __init__(self, wl: Workload, sample_seqs, mode=0, min_budget=0, max_budget=0,
-                 max_answer_tokens=0, device="cuda", evict_every=1, literal_return=0):
+                 max_answer_tokens=0, device="cuda", evict_every=1, literal_return=0, budget_ratio=0.0):
         self.wl, self.seqs, self.dev = wl, list(sample_seqs), device
         ctx = wl.prompt + wl.think_steps + wl.answer_steps + 2
         self.gpu = CrystalKV(Config(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
                                     batch=wl.batch, budget_per_head=wl.budget_per_head, max_context=ctx,
                                     min_budget=min_budget, max_budget=max_budget,
                                     max_answer_tokens=max_answer_tokens, top_p=wl.top_p, lam=wl.lam, mode=mode,
-                                    evict_every=evict_every, literal_return=literal_return))
+                                    evict_every=evict_every, literal_return=literal_return, budget_ratio=budget_ratio))
         bph = wl.budget_per_head
         self.ora = Oracle(OracleConfig(n_layers=wl.n_layers, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
                                        batch=len(self.seqs), budget_per_head=bph, max_context=ctx,
                                        min_budget=min_budget or min(bph, max(16, bph // 8)),
                                        max_budget=max_budget or 4 * bph, top_p=wl.top_p, lam=wl.lam, mode=mode,
-                                       evict_every=evict_every, literal_return=literal_return))
+                                       evict_every=evict_every, literal_return=literal_return, budget_ratio=budget_ratio))
         self.rep = Report()
         self.t = wl.prompt - 1
         self._tie_seen = 0
         self._agreed = {}          # (layer, sample index, head) -> (records, time) of the last agreed state (time None: before the prefill's scoring pass)
         self._budget_at_agreement = {}
+        self._first_budget = wl.budget_per_head
         self._tie_times = {}       # (layer, sample index, head) -> times of hit-mask near-ties since then
 
     def close(self):
@@ -81,6 +82,7 @@ class LockStep:
         self.gpu.check()
         # the state before the scoring pass is known exactly: the prompt entries, CRF 0, tau = P - 1
         P = wl.prompt
+        self._first_budget = int(self.ora.get_budgets()[0, 0, 0])   # uniform at this point
         rec0 = np.stack([np.arange(P), np.zeros(P, dtype=np.int64), np.full(P, P - 1)], axis=1).astype(np.int32)
         for l in range(wl.n_layers):
             for si in range(len(self.seqs)):
@@ -162,7 +164,7 @@ class LockStep:
         k0, v0 = wl.keys(l, pos0, seqs=[s])[0, :, h], wl.values(l, pos0, seqs=[s])[0, :, h]
         q = wl.queries(l, steps, seqs=[s])[0, :, h * G:(h + 1) * G].contiguous()
         kn, vn = wl.keys(l, steps, seqs=[s])[0, :, h].contiguous(), wl.values(l, steps, seqs=[s])[0, :, h].contiguous()
-        budget = int(self._budget_at_agreement.get(key, wl.budget_per_head))
+        budget = int(self._budget_at_agreement.get(key, self._first_budget))
         # fewest flips first; the all-zero pattern is the oracle's own run, which already disagreed
         patterns = sorted(itertools.product((0, 1, 2, 3), repeat=len(times)), key=lambda p: sum(x != 0 for x in p))
         for pat in patterns[1:]:

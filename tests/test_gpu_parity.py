@@ -129,6 +129,46 @@ def test_rebudget_small_with_answer_stage():
     ls.close()
 
 
+@pytest.mark.parametrize("prompt,budget", [(256, 64), (1000, 250), (83, 53)])
+def test_prompt_far_longer_than_the_budget_needs_no_reserve(prompt, budget):
+    """A prompt of four times the budget with no answer reserve: the prompt is scored from the caller's
+    tensors and only the survivors of the one Algorithm 1 pass are stored, so the pool (sized for the
+    budget) is never exceeded; state and ownership against the oracle, then decode steps."""
+    wl = Workload(name=f"long{prompt}", seed=700 + prompt, n_layers=2, n_q_heads=10, n_kv_heads=2, batch=3,
+                  prompt=prompt, think_steps=30, budget_per_head=budget, outlier="flat", outlier_frac=0.05)
+    ls = LockStep(wl, [0, 2], max_budget=max(4 * budget, prompt))
+    ls.prefill()
+    ls.gpu.validate()
+    for h in range(2):
+        assert len(ls.gpu.get_retained(1, 2, h)) == budget
+    for _ in range(wl.think_steps):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
+def test_ratio_budgets_follow_the_context():
+    """Ratio budgets: the prompt's share at prefill (heads evict down to it), then Algorithm 2 over a
+    total that grows with the context at every reallocation; budgets, retained sets and CRF state
+    against the oracle."""
+    wl = Workload(name="ratio", seed=88, n_layers=3, n_q_heads=8, n_kv_heads=4, batch=3, prompt=96,
+                  think_steps=160, budget_per_head=96, rebudget_every=16, outlier="perhead", outlier_lo=0.01, outlier_hi=0.3)
+    ls = LockStep(wl, [0, 2], min_budget=4, max_budget=200, max_answer_tokens=80, budget_ratio=0.25)
+    ls.prefill()
+    assert (ls.gpu.get_budgets() == 24).all() and len(ls.gpu.get_retained(2, 2, 3)) == 24
+    totals = []
+    for s in range(wl.think_steps):
+        ls.step()
+        if (s + 1) % wl.rebudget_every == 0:
+            ls.rebudget()
+            totals.append(int(ls.gpu.get_budgets()[0].sum()))
+    assert totals == [min(96, (96 + 16 * (i + 1)) // 4) * 12 for i in range(10)]
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
 def test_fullkv_mode_is_plain_decode_attention():
     wl = Workload(name="full", seed=9, n_layers=2, n_q_heads=10, n_kv_heads=2, batch=2, prompt=100,
                   think_steps=60, budget_per_head=16)

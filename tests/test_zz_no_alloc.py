@@ -86,6 +86,30 @@ def test_static_check_after_a_larger_handle_used_the_array():
     ks.close()
 
 
+def test_both_checks_report_a_page_owned_twice():
+    """A page table edited from the host so that one head names a page of another: one page is
+    then owned twice and one not at all, and both entry points must say so (and agree).  The
+    handle is only validated and destroyed afterwards."""
+    wl = Workload(name="na_bad", seed=44, n_layers=2, n_q_heads=4, n_kv_heads=2, batch=2, prompt=40,
+                  think_steps=8, budget_per_head=64)
+    kv = _run(wl, 8)
+    assert _verdict(kv.validate)[0] == 0 and _verdict(kv.validate_static) == (0, (0, 0))
+    # head (layer 1, seq 1, head 0) owns pages 0..2 of its list (48 entries + the next arrival): its second
+    # page is replaced by the id the first head of the sequence holds first
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    victim = 0      # page ids are handed out in ascending order from 0 within a sequence
+    assert kv.lib.crystalkv_debug_set_page(kv._h, 1, 1, 0, 1, victim, stream) == 0
+    assert kv.lib.crystalkv_debug_set_page(kv._h, 1, 1, 0, 10 ** 6, 0, stream) == -1      # index out of range
+    assert kv.lib.crystalkv_debug_set_page(kv._h, 1, 1, 0, 0, 10 ** 9, stream) == -1      # page out of range
+    code, _ = _verdict(kv.validate)
+    assert code == -5
+    assert b"2 pages not owned exactly once" in kv.lib.crystalkv_last_error(kv._h)
+    counts = np.full(2, -1, dtype=np.int32)
+    rc = kv.lib.crystalkv_validate_static(kv._h, counts.ctypes.data_as(C.c_void_p), stream)
+    assert rc == -5 and tuple(counts) == (0, 2)
+    kv.close()
+
+
 def test_static_check_refuses_a_handle_beyond_its_array():
     """2**17 pool pages (16 entries each) is the limit; a handle with more is refused with EINVAL
     and a message that names the limit, and nothing is launched."""
