@@ -250,8 +250,7 @@ int crystalkv_validate(crystalkv_t* h, void* stream);
  * device-wide synchronisation a cudaMalloc / cudaFree pair implies.  This entry point does the
  * same check with its per-page counters in an array that is built into the library: it calls
  * no cudaMalloc, cudaFree or other allocating routine.  Like crystalkv_validate it copies its
- * verdict to the host and synchronises `stream`, so it is not a call for a stream that is
- * being captured.
+ * verdict to the host and synchronises `stream`.
  *
  *   counts_out_host  host int32[2] or NULL: [0] page ids or counts out of range, [1] pages not
  *                    owned exactly once (both 0 on a sound handle)

@@ -1,19 +1,21 @@
 // Decode attention of one layer (Section 2.2): the G queries of every kv head over its paged
 // cache, split-K over the warps of a persistent grid.
 //
-// The layer's launch plan (plan.cuh) gives every warp a run of 16-key groups, one piece per head
-// the run overlaps.  A group is one pool page: 16 entries (K row + V row each) in 8 KB, stored
-// so that the page, copied as it is into a ring stage by ONE bulk asynchronous copy, is read by
-// ldmatrix without bank conflicts.  A warp keeps its ring of STAGES pages full across piece
-// boundaries (the copies only need the cache, not the queries), waits for a stage on its
-// mbarrier, and runs both contractions on the tensor cores with keys on the MMA M dimension and
-// the (padded) query heads on N = 8:   S[16 keys x 8 heads] = K Q^T,   O^T[128 x 8 heads] += V^T P^T.
+// The layer's launch plan (plan.cuh) gives every warp its pieces: a piece is a range of the 16-key
+// groups of one head (usually one piece per warp; several whole heads when there are more heads
+// than warps).  A group is one pool page: 16 entries (K row + V row each) in 8 KB, stored so that
+// the page, copied as it is into a ring stage by ONE bulk asynchronous copy, is read by ldmatrix
+// without bank conflicts.  A warp keeps its ring of STAGES pages full across piece boundaries
+// (the copies only need the cache, not the queries), waits for a stage on its mbarrier, and runs
+// both contractions on the tensor cores with keys on the MMA M dimension and the (padded) query
+// heads on N = 8:   S[16 keys x 8 heads] = K Q^T,   O^T[128 x 8 heads] += V^T P^T.
 // A head that is one piece is written out directly; otherwise every piece publishes its
-// (m, l, O) partial and the warp whose partial completes the head merges them into `out`, after
-// it has finished its own run.  The arriving token is written into the head's hole (the place an
-// evicted entry left, or the end of the list) by the warp that streams that group.  The scaled
-// logits of the step are left in the scratch for the LRFU kernel, which marks hits from the
-// final softmax weights without reading the cache again.
+// (m, l, O) partial and the warp whose partial completes the head merges them into `out` (after
+// its own pieces, if it has more).  The arriving token is written into the head's hole (the place
+// an evicted entry left, or the end of the list) by the warp that streams that group.  The scaled
+// logits of the step are left in the scratch for the LRFU kernel, which marks hits from the final
+// softmax weights without reading the cache again; the lines of the metadata that kernel will
+// read are asked into L2 on the way.
 #pragma once
 #include "common.cuh"
 

@@ -422,6 +422,71 @@ def test_a_smaller_handle_created_later_leaves_a_larger_one_working():
     ls.close()
 
 
+def test_a_handle_rebuilt_from_exports_continues_like_the_original():
+    """Every head exported (records and K/V rows) after 120 steps with two reallocations, the handle
+    destroyed, a fresh handle rebuilt by import alone (no prefill), 60 more steps on both the rebuilt
+    handle and an uninterrupted twin: outputs, budgets and state bit for bit, ownership sound."""
+    from paper_2601_16986_b200 import Config, CrystalKV, CrystalKVError
+    wl = Workload(name="ckpt", seed=123, n_layers=3, n_q_heads=10, n_kv_heads=2, batch=2, prompt=70,
+                  think_steps=180, budget_per_head=64, rebudget_every=50, outlier="perhead", outlier_lo=0.01, outlier_hi=0.3)
+    cfg = Config(n_layers=3, n_q_heads=10, n_kv_heads=2, batch=2, budget_per_head=64, max_context=300, min_budget=8)
+
+    def fresh(prefill=True):
+        kv = CrystalKV(cfg)
+        if prefill:
+            for l in range(3):
+                k, v = wl.prompt_kv(l, device="cuda")
+                kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], device="cuda")[:, 0].contiguous())
+        return kv
+
+    def run(kv, s0, s1):
+        outs = []
+        for s in range(s0, s1):
+            for l in range(3):
+                outs.append(kv.decode_step(l, *wl.step_inputs(l, wl.prompt + s, device="cuda")).clone())
+            if (s + 1) % wl.rebudget_every == 0:
+                kv.rebudget()
+        return outs
+
+    a, twin = fresh(), fresh()
+    run(a, 0, 120); run(twin, 0, 120)
+    budgets = a.get_budgets()
+    saved = {}
+    for l in range(3):
+        for b in range(2):
+            for h in range(2):
+                rec = a.export_state(l, b, h)
+                k, v = a.export_kv(l, b, h)
+                pos = rec[:, 0].tolist()
+                assert torch.equal(k, wl.keys(l, pos, seqs=[b])[0, :, h]) and torch.equal(v, wl.values(l, pos, seqs=[b])[0, :, h])
+                saved[(l, b, h)] = (rec, k.contiguous(), v.contiguous())
+    t = a.time(0)
+    a.close()
+    c = fresh(prefill=False)
+    with pytest.raises(CrystalKVError):                       # a record after the layer's time
+        rec, k, v = saved[(0, 0, 0)]
+        bad = rec.copy(); bad[0, 2] = t + 5
+        c.import_state(0, 0, 0, bad, k, v, int(budgets[0, 0, 0]), t)
+    for (l, b, h), (rec, k, v) in saved.items():
+        perm = np.random.default_rng(l * 7 + b * 3 + h).permutation(len(rec))     # any order is accepted
+        c.import_state(l, b, h, rec[perm], k[torch.as_tensor(perm)].contiguous(), v[torch.as_tensor(perm)].contiguous(),
+                       int(budgets[b, l, h]), t)
+    with pytest.raises(CrystalKVError):                       # the layer is at time t now
+        rec, k, v = saved[(1, 1, 1)]
+        c.import_state(1, 1, 1, rec, k, v, 0, t + 1)
+    c.check(); c.validate()
+    assert (c.get_budgets() == budgets).all()
+    oc, ot = run(c, 120, 180), run(twin, 120, 180)
+    assert all(torch.equal(x, y) for x, y in zip(oc, ot))
+    assert (c.get_budgets() == twin.get_budgets()).all()
+    for l in range(3):
+        for b in range(2):
+            for h in range(2):
+                assert (c.export_state(l, b, h) == twin.export_state(l, b, h)).all()
+    for kv in (c, twin):
+        kv.check(); kv.validate(); kv.close()
+
+
 # ------------------------------------------------------------------ error paths on a live handle
 @pytest.mark.parametrize("W,prompt,budget", [(1, 83, 53), (8, 83, 53), (32, 200, 96), (40, 40, 64), (16, 300, 256)])
 def test_observation_window_prefill(W, prompt, budget):
