@@ -102,6 +102,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
   }
 }
 
+// Named barriers 1..NW: the warps that hold the pieces of one head meet there.
+__device__ __forceinline__ void bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;\n" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int nthreads) {
+  asm volatile("bar.arrive %0, %1;\n" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 constexpr float LAZY = 8.0f;   // the running maximum (log2 domain) may trail the true one by this much
 
 // The merge of HB heads over at most PB pieces in one round of loads: every lane loads the
@@ -324,6 +332,11 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
     const unsigned g_u = (unsigned)(n_tot + GRP - 1) / GRP;
     const int lo = (int)(g_u * (unsigned)piece / (unsigned)npieces), hi = (int)(g_u * (unsigned)(piece + 1) / (unsigned)npieces);
     const int hole = p.append ? __ldg(st.hole + uid) : -1;   // where the arriving token goes
+    // A head whose pieces all belong to warps of this CTA, each warp holding nothing else, is merged
+    // through shared memory (the plan hands consecutive pieces to consecutive warps).
+    const int first_w = w - piece;
+    const bool local = npieces > 1 && range.y - range.x == 1 && first_w >= 0 && first_w + npieces <= NW &&
+                       pi - piece == (int)blockIdx.x * NW + first_w;
     // the G queries as B fragments, running softmax state, O^T accumulators
     uint32_t qb[8][2];
     {
@@ -348,6 +361,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
         if (lane == 0) atomicOr(st.errword, ERR_COPY_TIMEOUT);
         for (int s = 0; s < STAGES; ++s)
           if (s != csi) mbar_wait_bounded(bar0 + s * 8, (phases >> s) & 1u);
+        if (local) bar_arrive(1 + first_w, 32 * npieces);   // the head's other warps must not wait for this one
         return;
       }
       phases ^= 1u << csi;
@@ -467,6 +481,59 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
       if (gid == 0 && p.track) {   // reference point and normaliser of the step's softmax, for the LRFU kernel
         if (h0 < G) { p.sc.mfin[u * (2 * QH) + h0] = m0; p.sc.mfin[u * (2 * QH) + QH + h0] = ls0; }
         if (h1 < G) { p.sc.mfin[u * (2 * QH) + h1] = m1; p.sc.mfin[u * (2 * QH) + QH + h1] = ls1; }
+      }
+      continue;
+    }
+    if (local) {
+      // ---- the piece's partial goes into this warp's ring (idle by now: its only piece is done);
+      // after a barrier of the head's warps each of them merges a share of the query heads
+      constexpr int HS = HD + 4;   // row stride that spreads the four head pairs of a store over the banks
+      constexpr int WSTRIDE = STAGES * PAGE_BYTES;
+      float* mine = reinterpret_cast<float*>(smem + w * WSTRIDE);
+      if (gid == 0) {
+        *reinterpret_cast<float2*>(mine + 2 * tig) = make_float2(m0, m1);
+        *reinterpret_cast<float2*>(mine + 8 + 2 * tig) = make_float2(ls0, ls1);
+      }
+      {
+        float* po = mine + 16 + gid;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          if (h0 < G) { po[h0 * HS + 16 * mt] = o[mt][0]; po[h0 * HS + 16 * mt + 8] = o[mt][2]; }
+          if (h1 < G) { po[h1 * HS + 16 * mt] = o[mt][1]; po[h1 * HS + 16 * mt + 8] = o[mt][3]; }
+        }
+      }
+      bar_sync(1 + first_w, 32 * npieces);
+      const unsigned char* base = smem + first_w * WSTRIDE;
+      for (int g = piece; g < G; g += npieces) {
+        float pm[NW], pl[NW];
+        float4 v[NW];
+        float m = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < NW; ++j) {
+          const float* pp = reinterpret_cast<const float*>(base + (j < npieces ? j : 0) * WSTRIDE);
+          pm[j] = (j < npieces) ? pp[g] : -INFINITY;
+          pl[j] = (j < npieces) ? pp[8 + g] : 0.f;
+          v[j] = *reinterpret_cast<const float4*>(pp + 16 + g * HS + lane * 4);
+          m = fmaxf(m, pm[j]);
+        }
+        float L = 0.f;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < NW; ++j) {
+          const float c = (pm[j] > -INFINITY) ? ex2(pm[j] - m) : 0.f;
+          L = fmaf(pl[j], c, L);
+          a.x = fmaf(v[j].x, c, a.x); a.y = fmaf(v[j].y, c, a.y);
+          a.z = fmaf(v[j].z, c, a.z); a.w = fmaf(v[j].w, c, a.w);
+        }
+        const float iv = 1.0f / L;
+        uint2 pk;
+        pk.x = pack_bf16(a.x * iv, a.y * iv);
+        pk.y = pack_bf16(a.z * iv, a.w * iv);
+        *reinterpret_cast<uint2*>(p.out + ((size_t)(u * G + g)) * HD + lane * 4) = pk;
+        if (lane == 0 && p.track) {
+          p.sc.mfin[u * (2 * QH) + g] = m;
+          p.sc.mfin[u * (2 * QH) + QH + g] = L;
+        }
       }
       continue;
     }

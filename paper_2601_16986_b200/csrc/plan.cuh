@@ -78,14 +78,15 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
       for (int j = 0; j < k; ++j) pl.desc[start + j] = make_int4(u, j, k, 0);
     }
   }
-  // ---- which warp takes which pieces: piece i goes to CTA i % grid, warp i / grid; with more
-  // pieces than warps every warp takes a run of consecutive pieces
+  // ---- which warp takes which pieces: consecutive pieces go to consecutive warps, so that most
+  // heads have all their pieces in one CTA and are merged in its shared memory (with fewer pieces
+  // than warps the last CTAs stay idle); with more pieces than warps every warp takes a run of
+  // consecutive pieces
   const int per = (pieces + nWarps - 1) / max(nWarps, 1);
   for (int pw = tid; pw < nWarps; pw += NT) {
     int2 r = make_int2(0, 0);
     if (pieces <= nWarps) {
-      const int i = (pw % NW) * grid + pw / NW;
-      if (i < pieces) r = make_int2(i, i + 1);
+      if (pw < pieces) r = make_int2(pw, pw + 1);
     } else {
       const int i0 = min(pieces, pw * per);
       r = make_int2(i0, min(pieces, i0 + per));
