@@ -282,6 +282,19 @@ int crystalkv_validate_static(crystalkv_t* h, int32_t* counts_out_host, void* st
 int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, int32_t index,
                              int32_t page, void* stream);
 
+/*
+ * Test hook (the paper has no counterpart): copies the launch plan of a layer's next attention
+ * kernel to the host.  hdr_host[4] = {pieces, groups (pages of 16 keys) over all heads, warps the
+ * plan is made for, 1 when it is for a decode step}; wrange_host[2 w], [2 w + 1] = the pieces
+ * [first, end) that warp w of the grid (CTA w / 8) streams, for w < hdr[2]; desc_host[4 i ..] =
+ * {head index seq * n_kv_heads + kv_head, j, k, together} of piece i: the j-th of the head's k
+ * pieces, `together` = 1 when the k pieces sit in consecutive warps of one CTA.  warps_cap and
+ * pieces_cap are the capacities of the two arrays in warps and in pieces; EINVAL unless
+ * warps_cap >= 8 x SMs and pieces_cap >= 8 x SMs + batch x n_kv_heads.  Synchronises `stream`.
+ */
+int crystalkv_debug_get_plan(crystalkv_t* h, int layer, int32_t* hdr_host, int32_t* wrange_host,
+                             int32_t warps_cap, int32_t* desc_host, int32_t pieces_cap, void* stream);
+
 const char* crystalkv_strerror(int code);
 const char* crystalkv_last_error(crystalkv_t* h);
 

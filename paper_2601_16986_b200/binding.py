@@ -100,6 +100,7 @@ def load_library():
     lib.crystalkv_validate.argtypes = [vp, vp]
     lib.crystalkv_validate_static.argtypes = [vp, vp, vp]
     lib.crystalkv_debug_set_page.argtypes = [vp, i32, i32, i32, C.c_int32, C.c_int32, vp]
+    lib.crystalkv_debug_get_plan.argtypes = [vp, i32, vp, vp, C.c_int32, vp, C.c_int32, vp]
     lib.crystalkv_strerror.argtypes = [i32]
     lib.crystalkv_strerror.restype = C.c_char_p
     lib.crystalkv_last_error.argtypes = [vp]
@@ -257,6 +258,19 @@ class CrystalKV:
 
     def validate(self):
         self._ck(self.lib.crystalkv_validate(self._h, _stream()))
+
+    def debug_plan(self, layer: int):
+        """Launch plan of the layer's next attention kernel (test hook): hdr int32[4], wrange
+        int32[warps, 2], desc int32[warps + heads, 4] as the header describes them."""
+        warps = 8 * torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+        heads = self.cfg.batch * self.cfg.n_kv_heads
+        hdr = np.zeros(4, dtype=np.int32)
+        wrange = np.zeros((warps, 2), dtype=np.int32)
+        desc = np.zeros((warps + heads, 4), dtype=np.int32)
+        vp = C.c_void_p
+        self._ck(self.lib.crystalkv_debug_get_plan(self._h, layer, hdr.ctypes.data_as(vp), wrange.ctypes.data_as(vp), warps,
+                                                   desc.ctypes.data_as(vp), warps + heads, _stream()))
+        return hdr, wrange, desc
 
     def validate_static(self) -> np.ndarray:
         """The same check without any device allocation (scratch built into the library; at

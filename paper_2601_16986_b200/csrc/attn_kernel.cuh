@@ -332,11 +332,10 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
     const unsigned g_u = (unsigned)(n_tot + GRP - 1) / GRP;
     const int lo = (int)(g_u * (unsigned)piece / (unsigned)npieces), hi = (int)(g_u * (unsigned)(piece + 1) / (unsigned)npieces);
     const int hole = p.append ? __ldg(st.hole + uid) : -1;   // where the arriving token goes
-    // A head whose pieces all belong to warps of this CTA, each warp holding nothing else, is merged
-    // through shared memory (the plan hands consecutive pieces to consecutive warps).
+    // A head whose pieces all belong to consecutive warps of this CTA, each warp holding nothing else
+    // (the plan marks it), is merged through shared memory.
     const int first_w = w - piece;
-    const bool local = npieces > 1 && range.y - range.x == 1 && first_w >= 0 && first_w + npieces <= NW &&
-                       pi - piece == (int)blockIdx.x * NW + first_w;
+    const bool local = dd.w != 0 && npieces > 1 && range.y - range.x == 1 && first_w >= 0 && first_w + npieces <= NW;
     // the G queries as B fragments, running softmax state, O^T accumulators
     uint32_t qb[8][2];
     {

@@ -1051,6 +1051,25 @@ int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, in
   return CRYSTALKV_OK;
 }
 
+int crystalkv_debug_get_plan(crystalkv_t* h, int layer, int32_t* hdr_host, int32_t* wrange_host, int32_t warps_cap,
+                             int32_t* desc_host, int32_t pieces_cap, void* stream) {
+  if (!h) return CRYSTALKV_EINVAL;
+  if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");
+  if (layer < 0 || layer >= h->cfg.n_layers || !hdr_host || !wrange_host || !desc_host)
+    return fail(h, CRYSTALKV_EINVAL, "layer out of range or a NULL output");
+  const int nWarps = h->grid * NW;
+  if (warps_cap < nWarps || pieces_cap < nWarps + h->U) return fail(h, CRYSTALKV_EINVAL, "output arrays too small for the plan");
+  ON_DEVICE(h);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (int jr = join_side(h, s)) return jr;
+  const Plan& pl = h->plans[layer];
+  CK(h, cudaMemcpyAsync(hdr_host, pl.hdr, 4 * sizeof(int), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaMemcpyAsync(wrange_host, pl.wrange, (size_t)nWarps * sizeof(int2), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaMemcpyAsync(desc_host, pl.desc, (size_t)(nWarps + h->U) * sizeof(int4), cudaMemcpyDeviceToHost, s));
+  CK(h, cudaStreamSynchronize(s));
+  return CRYSTALKV_OK;
+}
+
 int crystalkv_join(crystalkv_t* h, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;
   if (h->cuda_dead) return fail(h, CRYSTALKV_ECUDA, "an earlier CUDA error is sticky for this handle");

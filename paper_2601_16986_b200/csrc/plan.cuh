@@ -16,12 +16,45 @@
 
 namespace ckv {
 
-// Called by all NT threads of one CTA.  `gs` is shared memory for U + 1 ints, `red` for NW + 1.
+// CTAs a set of heads needs when the pieces of a head have to sit in consecutive warps of one CTA:
+// `full` CTAs are taken whole (eight pieces of a head with eight or more), cnt[s] runs of s < 8
+// pieces are packed best fit, longest first.  A run goes to the open CTA with the fewest free
+// warps that still holds it, so a CTA with c free warps takes c / s runs of length s one after the
+// other: the loop below moves whole classes of CTAs at once and counts exactly what the
+// run-by-run placement in write_plan() does.
+__device__ __forceinline__ int ctas_needed(int full, const int (&cnt)[8]) {
+  int open[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // open[c]: CTAs with c free warps
+  int ctas = full;
+#pragma unroll
+  for (int s = 7; s >= 1; --s) {
+    int n = cnt[s];
+#pragma unroll
+    for (int c = s; c <= 8; ++c) {
+      const int q = c / s;                              // runs one such CTA takes
+      const int have = (c == 8) ? (n + q - 1) / q : open[c];   // fresh CTAs are not counted in open[]
+      const int nb = min(have, n / q);                  // CTAs filled with q runs
+      int left = c - q * s;
+      if (c == 8) ctas += nb; else open[c] -= nb;
+      open[left] += nb;
+      n -= nb * q;
+      if (n > 0 && n < q && have > nb) {                // one more takes the rest
+        if (c == 8) ++ctas; else --open[c];
+#pragma unroll
+        for (int nn = 1; nn < 8; ++nn)
+          if (nn < q && n == nn) open[c - nn * s] += 1;
+        n = 0;
+      }
+    }
+  }
+  return ctas;
+}
+
+// Called by all NT threads of one CTA.  `gs` is shared memory for U + 1 ints, `red` for 320.
 // append: the plan is for a decode step (every head one entry longer than now); n_limit > 0: for
 // a scoring pass over the first n_limit entries of every head.
 __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int layer, int append, int n_limit, int nWarps,
                                         int grid, int* gs, int* red) {
-  const int U = st.batch * st.H, tid = threadIdx.x;
+  const int U = st.batch * st.H, tid = threadIdx.x, lane = tid & 31;
   // ---- groups per head
   int mine = 0, gmax = 0, empty = 0;
   for (int u = tid; u < U; u += NT) {
@@ -39,7 +72,7 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) gmax = max(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
   __syncthreads();
-  if ((tid & 31) == 0) red[tid >> 5] = gmax;
+  if (lane == 0) red[tid >> 5] = gmax;
   __syncthreads();
   for (int x = 0; x < NW; ++x) gmax = max(gmax, red[x]);
   empty = __syncthreads_or(empty);
@@ -47,10 +80,53 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
     if (tid == 0) atomicOr(st.errword, ERR_PLAN);
     Gtot = 0;
   }
-  // ---- the piece bound T: the smallest for which sum ceil(g_u / T) <= nWarps (none when there
-  // are more heads than warps: one piece per head then)
+  // ---- the piece bound T.  Heads are cut into ceil(g_u / T) pieces; the smallest T is wanted for
+  // which all heads can be placed with every head's pieces inside one CTA (such a head is merged in
+  // shared memory; one that straddles CTAs goes through global memory and a ticket, which costs the
+  // launch two to three microseconds at its end).  32 candidates are tried at once: warp x counts the
+  // runs of every length over the heads u = x mod 8, lane c for T0 + c; warp 0 then packs them.
   int T = 0x7fffffff;
-  if (Gtot > 0 && U <= nWarps) {
+  bool packed = false;
+  int* hist = red + 16;   // [32][4]: counts of two run lengths per word, 16 bits each (U < 65536)
+  if (Gtot > 0 && U <= nWarps && grid * NW == nWarps && grid <= 256 && nWarps < 4096) {
+    const int T0 = max(max(1, (Gtot + nWarps - 1) / nWarps), min(GMIN, gmax));   // pieces shorter than GMIN groups
+                                                                                // cost more in starts and merges than they gain
+    for (int round = 0; round < 4 && !packed; ++round) {
+      const int Tc = T0 + round * 32 + lane;
+      if (tid < 128) hist[tid] = 0;
+      __syncthreads();
+      unsigned h4[4] = {0u, 0u, 0u, 0u};
+      for (int u = tid >> 5; u < U; u += NW) {
+        const int k = (gs[u] + Tc - 1) / Tc;
+        const int r = k & 7;   // 0: nothing beyond whole CTAs
+#pragma unroll
+        for (int x = 0; x < 4; ++x) h4[x] += ((x > 0 && r == 2 * x) ? 1u : 0u) + ((r == 2 * x + 1) ? 0x10000u : 0u);
+        h4[0] += (unsigned)(k >> 3);   // the low half of word 0 counts whole CTAs (there is no run of length 0)
+      }
+#pragma unroll
+      for (int x = 0; x < 4; ++x) atomicAdd(reinterpret_cast<unsigned*>(hist) + lane * 4 + x, h4[x]);
+      __syncthreads();
+      int ok = 0;
+      if (tid < 32) {
+        int cnt[8];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const unsigned v = (unsigned)hist[lane * 4 + x];
+          cnt[2 * x] = (int)(v & 0xffffu);
+          cnt[2 * x + 1] = (int)(v >> 16);
+        }
+        const int full = cnt[0];
+        ok = ctas_needed(full, cnt) <= grid;
+        const unsigned m = __ballot_sync(0xffffffffu, ok);
+        if (lane == 0) red[0] = m ? T0 + round * 32 + (__ffs(m) - 1) : -1;
+      }
+      __syncthreads();
+      if (red[0] > 0) { T = red[0]; packed = true; }
+      __syncthreads();
+    }
+  }
+  if (!packed && Gtot > 0 && U <= nWarps) {
+    // fallback: the smallest T for which sum ceil(g_u / T) <= nWarps, heads laid over the warps end to end
     int lo = max(1, (Gtot + nWarps - 1) / nWarps), hi = max(lo, gmax);   // feasible at hi: one piece per head
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
@@ -61,7 +137,7 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
       __syncthreads();
       if (tot <= nWarps) hi = mid; else lo = mid + 1;
     }
-    T = max(lo, min(GMIN, gmax));   // pieces shorter than GMIN groups cost more in starts and merges than they gain
+    T = max(lo, min(GMIN, gmax));
   }
   // ---- pieces per head, their prefix sums, the descriptors
   int pieces = 0;
@@ -75,28 +151,94 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
     if (u < U) {
       pl.npc[u] = k;
       pl.gplan[u] = g;
-      for (int j = 0; j < k; ++j) pl.desc[start + j] = make_int4(u, j, k, 0);
+      // the last word: 1 when the head's k pieces sit in consecutive warps of one CTA, each warp with
+      // nothing else to stream
+      const int together = k > 1 && (packed ? k <= NW : (start & (NW - 1)) + k <= NW);
+      for (int j = 0; j < k; ++j) pl.desc[start + j] = make_int4(u, j, k, together);
+      if (packed) gs[u] = (start << 12) | k;
     }
   }
-  // ---- which warp takes which pieces: consecutive pieces go to consecutive warps, so that most
-  // heads have all their pieces in one CTA and are merged in its shared memory (with fewer pieces
-  // than warps the last CTAs stay idle); with more pieces than warps every warp takes a run of
-  // consecutive pieces
-  const int per = (pieces + nWarps - 1) / max(nWarps, 1);
-  for (int pw = tid; pw < nWarps; pw += NT) {
-    int2 r = make_int2(0, 0);
-    if (pieces <= nWarps) {
-      if (pw < pieces) r = make_int2(pw, pw + 1);
-    } else {
-      const int i0 = min(pieces, pw * per);
-      r = make_int2(i0, min(pieces, i0 + per));
+  if (packed) {
+    for (int pw = tid; pw < nWarps; pw += NT) pl.wrange[pw] = make_int2(0, 0);
+    __syncthreads();
+    if (tid < 32) {
+      // every lane keeps the same books; the lanes share the stores
+      int* nxt = red + 16;   // [grid] next CTA in the list of its class
+      int next_cta = 0, over = 0;
+      for (int b0 = 0; b0 < U && !over; b0 += 32) {   // whole CTAs first
+        const int v = (b0 + lane < U) ? gs[b0 + lane] : 0;
+        unsigned m = __ballot_sync(0xffffffffu, (v & 4095) >= NW);
+        while (m) {
+          const int b = __ffs(m) - 1;
+          m &= m - 1;
+          const int vv = __shfl_sync(0xffffffffu, v, b);
+          const int start = vv >> 12, nw = ((vv & 4095) >> 3) * NW;
+          if (next_cta * NW + nw > nWarps) { over = 1; break; }
+          for (int x = lane; x < nw; x += 32) pl.wrange[next_cta * NW + x] = make_int2(start + x, start + x + 1);
+          next_cta += nw / NW;
+        }
+      }
+      int head[8] = {-1, -1, -1, -1, -1, -1, -1, -1};   // head[c]: first of the CTAs with c free warps
+#pragma unroll
+      for (int s = 7; s >= 1; --s) {
+        for (int b0 = 0; b0 < U && !over; b0 += 32) {
+          const int v = (b0 + lane < U) ? gs[b0 + lane] : 0;
+          unsigned m = __ballot_sync(0xffffffffu, (v & 7) == s);
+          while (m) {
+            const int b = __ffs(m) - 1;
+            m &= m - 1;
+            const int vv = __shfl_sync(0xffffffffu, v, b);
+            const int start = vv >> 12, k = vv & 4095;
+            int cta = -1, c = 8;
+#pragma unroll
+            for (int cc = s; cc <= 7; ++cc)
+              if (cta < 0 && head[cc] >= 0) {
+                cta = head[cc];
+                head[cc] = nxt[cta];
+                c = cc;
+              }
+            if (cta < 0) {
+              if (next_cta >= grid) { over = 1; break; }
+              cta = next_cta++;
+            }
+            const int left = c - s;
+#pragma unroll
+            for (int dd = 1; dd <= 7; ++dd)
+              if (left == dd) {
+                nxt[cta] = head[dd];
+                head[dd] = cta;
+              }
+            __syncwarp();
+            const int j0 = k - s;   // the pieces before these took whole CTAs
+            if (lane < s) pl.wrange[cta * NW + (NW - c) + lane] = make_int2(start + j0 + lane, start + j0 + lane + 1);
+          }
+        }
+      }
+      if (over && lane == 0) {   // cannot happen while ctas_needed() counts what this loop does; never leave half a plan
+        atomicOr(st.errword, ERR_PLAN);
+        nWarps = -1;
+      }
+      nWarps = __shfl_sync(0xffffffffu, nWarps, 0);
     }
-    pl.wrange[pw] = r;
+  } else {
+    // heads end to end: consecutive pieces go to consecutive warps; with more pieces than warps
+    // every warp takes a run of consecutive pieces
+    const int per = (pieces + nWarps - 1) / max(nWarps, 1);
+    for (int pw = tid; pw < nWarps; pw += NT) {
+      int2 r = make_int2(0, 0);
+      if (pieces <= nWarps) {
+        if (pw < pieces) r = make_int2(pw, pw + 1);
+      } else {
+        const int i0 = min(pieces, pw * per);
+        r = make_int2(i0, min(pieces, i0 + per));
+      }
+      pl.wrange[pw] = r;
+    }
   }
   if (tid == 0) {
     pl.hdr[0] = pieces;
     pl.hdr[1] = Gtot;
-    pl.hdr[2] = nWarps;
+    pl.hdr[2] = nWarps;   // (-1 after a failed placement: no launch accepts the plan)
     pl.hdr[3] = append;
   }
 }
@@ -106,7 +248,7 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
 __global__ void __launch_bounds__(NT) plan_kernel(State st, const Plan* plans, int layer0, int append, int n_limit,
                                                   int nWarps, int grid) {
   __shared__ int s_gs[MAX_UNITS_PER_CALL + 1];
-  __shared__ int s_red[NW + 1];
+  __shared__ int s_red[320];
   write_plan(st, plans[layer0 + blockIdx.x], layer0 + blockIdx.x, append, n_limit, nWarps, grid, s_gs, s_red);
 }
 

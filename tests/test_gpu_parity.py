@@ -203,6 +203,106 @@ def test_shrinking_one_budget_by_hand():
     ls.close()
 
 
+def _check_plan(kv, layer, lengths, n_kv_heads):
+    """Structure of a launch plan against the heads' lengths (entries before the arriving one)."""
+    hdr, wrange, desc = kv.debug_plan(layer)
+    pieces, groups, warps, append = (int(x) for x in hdr)
+    assert append == 1 and warps == wrange.shape[0]
+    g = {u: (n + 1 + 15) // 16 for u, n in lengths.items()}
+    assert groups == sum(g.values())
+    # pieces: head after head, j = 0 .. k - 1
+    i = 0
+    first = {}
+    for u in sorted(g):
+        k = int(desc[i, 2])
+        assert k >= 1
+        first[u] = i
+        for j in range(k):
+            assert tuple(desc[i + j, :3]) == (u, j, k), (u, j, desc[i + j])
+            assert desc[i + j, 3] == desc[i, 3]
+        i += k
+    assert i == pieces
+    # every piece belongs to exactly one warp
+    owner = np.full(pieces, -1)
+    for w in range(warps):
+        a, b = wrange[w]
+        assert 0 <= a <= b <= pieces
+        assert (owner[a:b] == -1).all()
+        owner[a:b] = w
+    assert (owner >= 0).all()
+    # heads marked `together`: consecutive warps of one CTA, nothing else in those warps
+    together = 0
+    for u in g:
+        k, i0 = int(desc[first[u], 2]), first[u]
+        if desc[i0, 3]:
+            ws = owner[i0:i0 + k]
+            assert (np.diff(ws) == 1).all() and ws[0] // 8 == ws[-1] // 8, (u, ws)
+            assert all(wrange[w][1] - wrange[w][0] == 1 for w in ws)
+            together += 1
+    # with at most one piece per warp, every head of two to eight pieces is placed that way
+    if pieces <= warps:
+        assert together == sum(1 for u in g if 2 <= desc[first[u], 2] <= 8)
+    longest = max(-(-g[u] // int(desc[first[u], 2])) for u in g)
+    return pieces, warps, together, longest, groups
+
+
+def test_launch_plans_keep_each_head_inside_one_cta():
+    """Heads of very different lengths in one launch: some need more than the eight warps of a
+    CTA (whole CTAs plus a shorter run elsewhere, merged through global memory), most need two to
+    eight (all in one CTA, merged in its shared memory), the shortest are one piece.  The plan is
+    checked as a structure, the outputs and the cache against the oracle."""
+    wl = Workload(name="mixed", seed=31, n_layers=2, n_q_heads=16, n_kv_heads=8, batch=2, prompt=1500,
+                  think_steps=12, budget_per_head=1600)
+    ls = LockStep(wl, [0, 1])
+    ls.prefill()
+    new = [1500, 1100, 700, 420, 300, 170, 100, 64, 50, 33, 17, 900, 1300, 250, 520, 75]
+    for seq in range(2):
+        for h in range(8):
+            b = new[seq * 8 + h]
+            for layer in range(2):
+                ls.gpu.set_budget(layer, seq, h, b)
+                ls.ora.set_budget(layer, seq, h, b)
+    ls.compare()
+    lengths = {seq * 8 + h: len(ls.gpu.get_retained(0, seq, h)) for seq in range(2) for h in range(8)}
+    assert sorted(lengths.values()) == sorted(new)
+    pieces, warps, together, longest, groups = _check_plan(ls.gpu, 0, lengths, 8)
+    assert together >= 6
+    assert longest <= max(4, 2 * -(-groups // warps))       # no warp streams much more than its share
+    for _ in range(12):
+        ls.step()
+    ls.gpu.check()
+    ls.assert_clean()
+    ls.close()
+
+
+def test_launch_plans_after_reallocations_are_all_inside_ctas():
+    """The 14B shape after reallocations: every head of two to eight pieces has them in one CTA."""
+    wl = WORKLOADS["cfg4_qwen14b"].scaled(n_layers=2, think_steps=300)
+    from paper_2601_16986_b200 import Config, CrystalKV
+    dev = torch.device("cuda", 0)
+    kv = CrystalKV(Config(n_layers=2, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, batch=wl.batch,
+                          budget_per_head=wl.budget_per_head, max_context=wl.prompt + 400, top_p=wl.top_p, lam=wl.lam))
+    for l in range(2):
+        k, v = wl.prompt_kv(l, device=dev)
+        kv.prefill(l, k, v, wl.queries(l, [wl.prompt - 1], device=dev)[:, 0].contiguous())
+    out = torch.empty(wl.batch, wl.n_q_heads, wl.head_dim, dtype=torch.bfloat16, device=dev)
+    for s in range(256):
+        pos = [wl.prompt + s]
+        for l in range(2):
+            kv.decode_step(l, wl.queries(l, pos, device=dev)[:, 0].contiguous(), wl.keys(l, pos, device=dev)[:, 0].contiguous(),
+                           wl.values(l, pos, device=dev)[:, 0].contiguous(), out)
+        if (s + 1) % 128 == 0:
+            kv.rebudget()
+    kv.check()
+    H = wl.n_kv_heads
+    for l in range(2):
+        lengths = {seq * H + h: len(kv.get_retained(l, seq, h)) for seq in range(wl.batch) for h in range(H)}
+        pieces, warps, together, longest, groups = _check_plan(kv, l, lengths, H)
+        assert together == len(lengths)          # (budgets of 300 and more: no head is a single piece here)
+        assert longest <= -(-groups // warps) * 1.25 + 1
+    kv.close()
+
+
 # ------------------------------------------------------------------ full-size shapes, sampled
 def _run_sampled(name, sample, n_steps, cmp_every, answer=0, max_answer=0):
     wl = WORKLOADS[name]
