@@ -87,52 +87,108 @@ def dram_traffic_from_profile(wl, args, entries_per_launch):
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 200 ms while a region runs."""
+    """SM clock, power and throttle reasons of one GPU while a region runs.  A child process reads
+    them through NVML every 2 ms for the whole run and stamps every sample with the host clock
+    (the timed region of a default run lasts tens of milliseconds, less than one period of
+    `nvidia-smi -lms`, and a thread of this process would wait for the launch loop's interpreter
+    lock); `with sampler:` marks the region, and the summary is over the samples inside it.
+    Where NVML cannot be loaded the child is `nvidia-smi -lms 50`."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+    CHILD = r"""
+import sys, time
+import pynvml as nv
+nv.nvmlInit()
+try:
+    hd = nv.nvmlDeviceGetHandleByUUID(sys.argv[1].encode()) if sys.argv[1] else nv.nvmlDeviceGetHandleByIndex(int(sys.argv[2]))
+except Exception:
+    hd = nv.nvmlDeviceGetHandleByIndex(int(sys.argv[2]))
+mx = nv.nvmlDeviceGetMaxClockInfo(hd, nv.NVML_CLOCK_SM)
+bits = (0x8, 0x40, 0x20, 0x4)
+print("ready", flush=True)
+i, mw = 0, 0
+while True:
+    sm = nv.nvmlDeviceGetClockInfo(hd, nv.NVML_CLOCK_SM)
+    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(hd)
+    if i % 8 == 0:
+        mw = nv.nvmlDeviceGetPowerUsage(hd)
+    i += 1
+    print(time.time(), sm, mx, mw / 1000.0, *["Active" if mask & b else "Not Active" for b in bits], sep=",", flush=True)
+    time.sleep(0.002)
+"""
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
-
-    def __enter__(self):
+        self.index, self.rows, self.proc, self.source, self.t0, self.t1 = index, [], None, None, None, None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+        except Exception:
+            uuid = ""
+        try:
+            self.proc = subprocess.Popen([sys.executable, "-c", self.CHILD, uuid, str(index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            if self.proc.stdout.readline().strip() != "ready":
+                raise OSError("NVML child did not start")
+            self.source = "nvml, 2 ms"
+        except Exception:
+            self._kill()
+            try:
+                self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
+                                              "--format=csv,noheader,nounits", "-lms", "50"],
+                                             stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                self.source = "nvidia-smi, 50 ms"
+            except OSError:
+                self.proc = None
+        if self.proc:
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
-        except OSError:
-            self.proc = None
-        return self
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            f = [x.strip() for x in line.split(",")]
+            if self.source and self.source.startswith("nvidia-smi"):
+                f = [str(time.time())] + f
+            self.rows.append(f)
+
+    def __enter__(self):
+        self.t0 = time.time()
+        return self
 
     def __exit__(self, *a):
+        self.t1 = time.time()
+
+    def _kill(self):
         if self.proc:
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=5)
             except Exception:
                 pass
+            self.proc = None
+
+    def close(self):
+        time.sleep(0.01)
+        self._kill()
 
     def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        sm, mx, pw, reasons = [], [], [], set()
+        for r in list(self.rows):
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
+                ts = float(r[0])
+                if self.t0 is None or not (self.t0 <= ts <= self.t1):
+                    continue
+                sm.append(float(r[1])); mx.append(float(r[2])); pw.append(float(r[3]))
             except (ValueError, IndexError):
                 continue
-            for n, v in zip(names, r[3:7]):
+            for n, v in zip(self.NAMES, r[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": self.source}
+        return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": max(mx), "power_w": statistics.median(pw),
+                "reasons": sorted(reasons), "samples": len(sm), "source": self.source,
+                "region_ms": (self.t1 - self.t0) * 1000.0}
 
 
 # ---------------------------------------------------------------------------------------
@@ -596,11 +652,15 @@ def main():
         launches["n"] = 0
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(stream)
+        if sampler:
+            sampler.__enter__()
         for s in range(s0, s1):
             one_step(s, inp, True)
         lib.crystalkv_join(h, sp)       # the last layers' LRFU kernels are inside the timed region
         ev1.record(stream)
         barrier()
+        if sampler:
+            sampler.__exit__()
         ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
         c1 = kv.get_counters()
         kv.check()
@@ -644,13 +704,14 @@ def main():
              "budget_min": int(budgets.min()), "budget_max": int(budgets.max())}
 
     # ---- warm-up and the timed steps, inputs resident before the region starts
+    clk = ClockSampler(local)
     main_in = StepInputs(n_all - s_prep)
     main_in.fill(s_prep)
     barrier()
     for s in range(s_prep, s_main):
         one_step(s, main_in, False)
-    with ClockSampler(local) as clk:
-        ms_total, roofline = timed_region(s_main, s_end, main_in)
+    ms_total, roofline = timed_region(s_main, s_end, main_in, sampler=clk)
+    clk.close()
     ms_rb = roofline["rebudget_ms_in_region"]
     ms_per_step = ms_total / args.steps
     value = world * args.steps / (ms_total / 1000.0)
