@@ -288,9 +288,11 @@ int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, in
  * plan is made for, 1 when it is for a decode step}; wrange_host[2 w], [2 w + 1] = the pieces
  * [first, end) that warp w of the grid (CTA w / 8) streams, for w < hdr[2]; desc_host[4 i ..] =
  * {head index seq * n_kv_heads + kv_head, j, k, together} of piece i: the j-th of the head's k
- * pieces, `together` = 1 when the k pieces sit in consecutive warps of one CTA.  warps_cap and
- * pieces_cap are the capacities of the two arrays in warps and in pieces; EINVAL unless
- * warps_cap >= 8 x SMs and pieces_cap >= 8 x SMs + batch x n_kv_heads.  Synchronises `stream`.
+ * pieces, `together` = 1 when the k pieces sit in consecutive warps of one CTA, 2 when they sit
+ * that way in runs of eight (pieces 8 r .. 8 r + 7 in the eight warps of one CTA) and one shorter
+ * run, 0 otherwise.  warps_cap and pieces_cap are the capacities of the two arrays in warps and
+ * in pieces; EINVAL unless warps_cap >= 8 x SMs and pieces_cap >= 8 x SMs + batch x n_kv_heads.
+ * Synchronises `stream`.
  */
 int crystalkv_debug_get_plan(crystalkv_t* h, int layer, int32_t* hdr_host, int32_t* wrange_host,
                              int32_t warps_cap, int32_t* desc_host, int32_t pieces_cap, void* stream);

@@ -334,8 +334,13 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
     const int hole = p.append ? __ldg(st.hole + uid) : -1;   // where the arriving token goes
     // A head whose pieces all belong to consecutive warps of this CTA, each warp holding nothing else
     // (the plan marks it), is merged through shared memory.
-    const int first_w = w - piece;
-    const bool local = dd.w != 0 && npieces > 1 && range.y - range.x == 1 && first_w >= 0 && first_w + npieces <= NW;
+    // (A head of more than eight pieces is placed in runs of eight, whole CTAs and one shorter run:
+    // every run is merged in its CTA, and only one partial per run goes through global memory.)
+    const bool runs = dd.w == 2;
+    const int jr = runs ? (piece & (NW - 1)) : piece;                       // this piece's place in its run
+    const int rl = runs ? min(NW, npieces - (piece & ~(NW - 1))) : npieces;   // pieces in the run
+    const int first_w = w - jr;
+    const bool local = dd.w != 0 && npieces > 1 && range.y - range.x == 1 && first_w >= 0 && first_w + rl <= NW;
     // the G queries as B fragments, running softmax state, O^T accumulators
     uint32_t qb[8][2];
     {
@@ -360,7 +365,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
         if (lane == 0) atomicOr(st.errword, ERR_COPY_TIMEOUT);
         for (int s = 0; s < STAGES; ++s)
           if (s != csi) mbar_wait_bounded(bar0 + s * 8, (phases >> s) & 1u);
-        if (local) bar_arrive(1 + first_w, 32 * npieces);   // the head's other warps must not wait for this one
+        if (local) bar_arrive(1 + first_w, 32 * rl);   // the run's other warps must not wait for this one
         return;
       }
       phases ^= 1u << csi;
@@ -501,17 +506,18 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
           if (h1 < G) { po[h1 * HS + 16 * mt] = o[mt][1]; po[h1 * HS + 16 * mt + 8] = o[mt][3]; }
         }
       }
-      bar_sync(1 + first_w, 32 * npieces);
+      bar_sync(1 + first_w, 32 * rl);
       const unsigned char* base = smem + first_w * WSTRIDE;
-      for (int g = piece; g < G; g += npieces) {
+      float* rpart = p.sc.partials + ((size_t)u * p.sc.pmax + (piece >> 3)) * PS;   // the run's partial (runs only)
+      for (int g = jr; g < G; g += rl) {
         float pm[NW], pl[NW];
         float4 v[NW];
         float m = -INFINITY;
 #pragma unroll
         for (int j = 0; j < NW; ++j) {
-          const float* pp = reinterpret_cast<const float*>(base + (j < npieces ? j : 0) * WSTRIDE);
-          pm[j] = (j < npieces) ? pp[g] : -INFINITY;
-          pl[j] = (j < npieces) ? pp[8 + g] : 0.f;
+          const float* pp = reinterpret_cast<const float*>(base + (j < rl ? j : 0) * WSTRIDE);
+          pm[j] = (j < rl) ? pp[g] : -INFINITY;
+          pl[j] = (j < rl) ? pp[8 + g] : 0.f;
           v[j] = *reinterpret_cast<const float4*>(pp + 16 + g * HS + lane * 4);
           m = fmaxf(m, pm[j]);
         }
@@ -524,6 +530,11 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
           a.x = fmaf(v[j].x, c, a.x); a.y = fmaf(v[j].y, c, a.y);
           a.z = fmaf(v[j].z, c, a.z); a.w = fmaf(v[j].w, c, a.w);
         }
+        if (runs) {   // the run's share of the head, not normalised
+          *reinterpret_cast<float4*>(rpart + 16 + g * HD + lane * 4) = a;
+          if (lane == 0) { rpart[g] = m; rpart[8 + g] = L; }
+          continue;
+        }
         const float iv = 1.0f / L;
         uint2 pk;
         pk.x = pack_bf16(a.x * iv, a.y * iv);
@@ -534,6 +545,19 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
           p.sc.mfin[u * (2 * QH) + QH + g] = L;
         }
       }
+      if (!runs) continue;
+      // every warp of the head counts itself once its share of its run's partial is written; the
+      // one that completes the count merges the runs
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) {
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;\n" : "=r"(old) : "l"(p.sc.ticket + u) : "memory");
+        last = (old == npieces - 1);
+        if (last) p.sc.ticket[u] = 0;
+      }
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) merge_head(p, u, (npieces + NW - 1) / NW, lane);
       continue;
     }
     // ---- publish the piece's partial and take a ticket

@@ -64,7 +64,7 @@ struct State {
 // correct when heads grow or shrink by a few entries; it is rewritten when a head's group count has
 // drifted from the one it was made for by an eighth (at least two), and after every reallocation.
 struct Plan {
-  int4* desc;        // [pd_cap] pieces, head after head: {head index u, piece j, pieces k of the head, 0}
+  int4* desc;        // [pd_cap] pieces, head after head: {head index u, piece j, pieces k of the head, how they are placed}
   int2* wrange;      // [warps] pieces [x, y) of the physical warp cta * NW + w
   int* npc;          // [U] pieces per head
   int* gplan;        // [U] groups per head the plan was made for

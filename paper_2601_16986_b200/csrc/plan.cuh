@@ -152,8 +152,8 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
       pl.npc[u] = k;
       pl.gplan[u] = g;
       // the last word: 1 when the head's k pieces sit in consecutive warps of one CTA, each warp with
-      // nothing else to stream
-      const int together = k > 1 && (packed ? k <= NW : (start & (NW - 1)) + k <= NW);
+      // nothing else to stream; 2 when they sit that way in runs of eight (whole CTAs) and one shorter run
+      const int together = k <= 1 ? 0 : (packed ? (k <= NW ? 1 : 2) : ((start & (NW - 1)) + k <= NW ? 1 : 0));
       for (int j = 0; j < k; ++j) pl.desc[start + j] = make_int4(u, j, k, together);
       if (packed) gs[u] = (start << 12) | k;
     }

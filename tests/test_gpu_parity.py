@@ -230,18 +230,22 @@ def _check_plan(kv, layer, lengths, n_kv_heads):
         assert (owner[a:b] == -1).all()
         owner[a:b] = w
     assert (owner >= 0).all()
-    # heads marked `together`: consecutive warps of one CTA, nothing else in those warps
+    # heads marked `together`: consecutive warps of one CTA, nothing else in those warps (mark 1), or
+    # the same for every run of eight pieces and the shorter last run (mark 2)
     together = 0
     for u in g:
-        k, i0 = int(desc[first[u], 2]), first[u]
-        if desc[i0, 3]:
-            ws = owner[i0:i0 + k]
-            assert (np.diff(ws) == 1).all() and ws[0] // 8 == ws[-1] // 8, (u, ws)
-            assert all(wrange[w][1] - wrange[w][0] == 1 for w in ws)
+        k, i0, mark = int(desc[first[u], 2]), first[u], int(desc[first[u], 3])
+        if mark:
+            assert (mark == 1) == (k <= 8)
+            for r0 in range(0, k, 8):
+                ws = owner[i0 + r0:i0 + min(k, r0 + 8)]
+                assert (np.diff(ws) == 1).all() and ws[0] // 8 == ws[-1] // 8, (u, ws)
+                assert k <= 8 or r0 + 8 > k or ws[0] % 8 == 0
+                assert all(wrange[w][1] - wrange[w][0] == 1 for w in ws)
             together += 1
-    # with at most one piece per warp, every head of two to eight pieces is placed that way
+    # with at most one piece per warp, every head of two or more pieces is placed that way
     if pieces <= warps:
-        assert together == sum(1 for u in g if 2 <= desc[first[u], 2] <= 8)
+        assert together == sum(1 for u in g if desc[first[u], 2] >= 2)
     longest = max(-(-g[u] // int(desc[first[u], 2])) for u in g)
     return pieces, warps, together, longest, groups
 
