@@ -223,7 +223,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
   if (tid < NW * STAGES) mbar_init(bars_u32 + tid * 8, 1);
   asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");   // made visible to the copy engine
   __syncthreads();
-  const int2 range = __ldg(p.plan.wrange + blockIdx.x * NW + w);   // (requested together with the header)
+  const int4 range = __ldg(p.plan.wrange + blockIdx.x * NW + w);   // (requested together with the header)
   if (__ldg(p.plan.hdr + 2) != (int)gridDim.x * NW || __ldg(p.plan.hdr + 3) != p.append) {   // a plan made for another launch
     if (tid == 0 && blockIdx.x == 0) atomicOr(st.errword, ERR_PLAN);
     return;
@@ -253,8 +253,10 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
     if (p.n_limit > 0) n = min(n, p.n_limit);
     return n + p.append;
   };
-  auto open_piece = [&](int pi) {
-    const int4 dd = __ldg(p.plan.desc + pi);
+  // the descriptor of the warp's first piece came with its range
+  const int4 dd_first = range.z >= 0 ? make_int4(range.z, range.w & 4095, (range.w >> 12) & 4095, range.w >> 24)
+                                     : __ldg(p.plan.desc + range.x);
+  auto open_piece = [&](int pi, const int4 dd) {
     const int u = dd.x;
     f_seq = u / st.H;
     f_ntot = entries_of(u);
@@ -289,7 +291,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
     if (f_next == f_hi) {
       f_pi = (f_pi + 1 < range.y) ? f_pi + 1 : -1;
       if (f_pi < 0) return false;
-      open_piece(f_pi);
+      open_piece(f_pi, __ldg(p.plan.desc + f_pi));
     }
     if (f_next - idbase >= 32) { idbase = f_next; ids = (f_next + lane < f_hi) ? __ldg(pt + f_next + lane) : 0; }
     const int page = __shfl_sync(0xffffffffu, ids, f_next - idbase);
@@ -311,7 +313,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
     fsi = (fsi + 1 == STAGES) ? 0 : fsi + 1;
     return true;
   };
-  open_piece(f_pi);
+  open_piece(f_pi, dd_first);
 #pragma unroll 1
   for (int s = 0; s < STAGES; ++s) fetch_next();
   // everything above reads only the cache, its lists and the plan; the call's inputs (q, the
@@ -324,7 +326,7 @@ __global__ void __maxnreg__(160) attn_kernel(const DecodeParams p) {   // (160 r
   while (fq_head != fq_tail) {
     const int pi = fifo[fq_head & (FIFO - 1)];
     ++fq_head;
-    const int4 dd = __ldg(p.plan.desc + pi);
+    const int4 dd = pi == range.x ? dd_first : __ldg(p.plan.desc + pi);
     const int u = dd.x, piece = dd.y, npieces = dd.z;
     const int seq = u / st.H;
     const int uid = (seq * st.L + p.layer) * st.H + (u % st.H);

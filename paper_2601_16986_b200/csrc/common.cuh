@@ -65,7 +65,9 @@ struct State {
 // drifted from the one it was made for by an eighth (at least two), and after every reallocation.
 struct Plan {
   int4* desc;        // [pd_cap] pieces, head after head: {head index u, piece j, pieces k of the head, how they are placed}
-  int2* wrange;      // [warps] pieces [x, y) of the physical warp cta * NW + w
+  int4* wrange;      // [warps] pieces [x, y) of the physical warp cta * NW + w; z, w: the descriptor of piece x
+                     // packed (z = head index, w = j | k << 12 | placement << 24) so that a warp starts without
+                     // a second dependent read, or z = -1: read desc[x]
   int* npc;          // [U] pieces per head
   int* gplan;        // [U] groups per head the plan was made for
   int* hdr;          // [4] pieces in total, groups in total, warps the plan was made for, append it was made for

@@ -482,7 +482,7 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   // launch plans, one per layer: at most one piece per warp and one more per head
   {
     const int nWarps = h->grid * NW, pd_cap = nWarps + h->U;
-    int4* desc = nullptr; int2* wr = nullptr; int *npc = nullptr, *gpl = nullptr, *hdr = nullptr;
+    int4* desc = nullptr; int4* wr = nullptr; int *npc = nullptr, *gpl = nullptr, *hdr = nullptr;
     DA(&desc, (size_t)c.n_layers * pd_cap);
     DA(&wr, (size_t)c.n_layers * nWarps);
     DA(&npc, (size_t)c.n_layers * h->U);
@@ -1064,9 +1064,11 @@ int crystalkv_debug_get_plan(crystalkv_t* h, int layer, int32_t* hdr_host, int32
   if (int jr = join_side(h, s)) return jr;
   const Plan& pl = h->plans[layer];
   CK(h, cudaMemcpyAsync(hdr_host, pl.hdr, 4 * sizeof(int), cudaMemcpyDeviceToHost, s));
-  CK(h, cudaMemcpyAsync(wrange_host, pl.wrange, (size_t)nWarps * sizeof(int2), cudaMemcpyDeviceToHost, s));
+  std::vector<int4> wr((size_t)nWarps);
+  CK(h, cudaMemcpyAsync(wr.data(), pl.wrange, (size_t)nWarps * sizeof(int4), cudaMemcpyDeviceToHost, s));
   CK(h, cudaMemcpyAsync(desc_host, pl.desc, (size_t)(nWarps + h->U) * sizeof(int4), cudaMemcpyDeviceToHost, s));
   CK(h, cudaStreamSynchronize(s));
+  for (int w = 0; w < nWarps; ++w) { wrange_host[2 * w] = wr[w].x; wrange_host[2 * w + 1] = wr[w].y; }
   return CRYSTALKV_OK;
 }
 

@@ -159,7 +159,7 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
     }
   }
   if (packed) {
-    for (int pw = tid; pw < nWarps; pw += NT) pl.wrange[pw] = make_int2(0, 0);
+    for (int pw = tid; pw < nWarps; pw += NT) pl.wrange[pw] = make_int4(0, 0, -1, 0);
     __syncthreads();
     if (tid < 32) {
       // every lane keeps the same books; the lanes share the stores
@@ -172,9 +172,10 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
           const int b = __ffs(m) - 1;
           m &= m - 1;
           const int vv = __shfl_sync(0xffffffffu, v, b);
-          const int start = vv >> 12, nw = ((vv & 4095) >> 3) * NW;
+          const int start = vv >> 12, kk = vv & 4095, nw = (kk >> 3) * NW;
           if (next_cta * NW + nw > nWarps) { over = 1; break; }
-          for (int x = lane; x < nw; x += 32) pl.wrange[next_cta * NW + x] = make_int2(start + x, start + x + 1);
+          for (int x = lane; x < nw; x += 32)
+            pl.wrange[next_cta * NW + x] = make_int4(start + x, start + x + 1, b0 + b, x | (kk << 12) | ((kk <= NW ? 1 : 2) << 24));
           next_cta += nw / NW;
         }
       }
@@ -210,7 +211,9 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
               }
             __syncwarp();
             const int j0 = k - s;   // the pieces before these took whole CTAs
-            if (lane < s) pl.wrange[cta * NW + (NW - c) + lane] = make_int2(start + j0 + lane, start + j0 + lane + 1);
+            if (lane < s)
+              pl.wrange[cta * NW + (NW - c) + lane] = make_int4(start + j0 + lane, start + j0 + lane + 1, b0 + b,
+                                                                (j0 + lane) | (k << 12) | ((k <= 1 ? 0 : (k <= NW ? 1 : 2)) << 24));
           }
         }
       }
@@ -225,12 +228,12 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
     // every warp takes a run of consecutive pieces
     const int per = (pieces + nWarps - 1) / max(nWarps, 1);
     for (int pw = tid; pw < nWarps; pw += NT) {
-      int2 r = make_int2(0, 0);
+      int4 r = make_int4(0, 0, -1, 0);
       if (pieces <= nWarps) {
-        if (pw < pieces) r = make_int2(pw, pw + 1);
+        if (pw < pieces) r = make_int4(pw, pw + 1, -1, 0);
       } else {
         const int i0 = min(pieces, pw * per);
-        r = make_int2(i0, min(pieces, i0 + per));
+        r = make_int4(i0, min(pieces, i0 + per), -1, 0);
       }
       pl.wrange[pw] = r;
     }
