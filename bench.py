@@ -268,22 +268,25 @@ def run_reference(args, wl):
 
 
 # ---------------------------------------------------------------------------------------
-def sweep_cell(wl, batch, budget, fullkv, context, steps, warmup, dev):
+def sweep_cell(wl, batch, budget, fullkv, context, steps, warmup, dev, ratio=0.0):
     """Steady-state decode of the 14B shape at one (batch, budget) cell, or of the full-cache
-    baseline with `context` entries per head; returns a dict for one table row."""
+    baseline with `context` entries per head; returns a dict for one table row.  ratio > 0: the
+    library's ratio rule sets the budgets (floor(ratio x tokens) per head on average) from a prompt
+    of `context` tokens; `budget` then only sizes the storage."""
     from paper_2601_16986_b200 import Config, CrystalKV, CrystalKVError, FULLKV, EVICT
     L, Hq, H, d = wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
-    P = context - 1 if fullkv else budget
+    P = context - 1 if fullkv else (context if ratio > 0 else budget)
     total = warmup + steps
     row = {"batch": batch, "budget": None if fullkv else budget, "mode": "fullkv" if fullkv else "crystal-kv",
            "entries_per_head": context if fullkv else budget + 1}
-    need_gb = batch * L * H * (P + total + 2) * 512 / 1e9
+    need_gb = batch * L * H * ((P if fullkv else budget) + total + 2) * 512 / 1e9
     if need_gb > 150:
         row["status"] = f"OOM: {need_gb:.0f} GB of K/V rows"
         return row
     try:
         kv = CrystalKV(Config(n_layers=L, n_q_heads=Hq, n_kv_heads=H, batch=batch, budget_per_head=budget,
-                              max_context=P + total + 2, mode=FULLKV if fullkv else EVICT, top_p=wl.top_p, lam=wl.lam))
+                              max_context=P + total + 2, mode=FULLKV if fullkv else EVICT, top_p=wl.top_p, lam=wl.lam,
+                              budget_ratio=ratio, max_budget=(P if ratio > 0 else 0)))   # (the prompt is scored in the heads' lists)
     except CrystalKVError as e:
         row["status"] = f"create failed: {e}"
         return row
@@ -295,11 +298,25 @@ def sweep_cell(wl, batch, budget, fullkv, context, steps, warmup, dev):
             for l in range(L):
                 kv.prefill(l, k, v, q)
             del k, v
+        elif ratio > 0:   # a long prompt: drawn sixteen sequences at a time (the generator's temporaries are 64-bit)
+            k = torch.empty(batch, P, H, d, dtype=torch.bfloat16, device=dev)
+            v = torch.empty_like(k)
+            for l in range(L):
+                for c0 in range(0, batch, 16):
+                    sq = list(range(c0, min(batch, c0 + 16)))
+                    k[c0:c0 + 16], v[c0:c0 + 16] = w.prompt_kv(l, seqs=sq, device=dev)
+                kv.prefill(l, k, v, w.queries(l, [P - 1], device=dev)[:, 0].contiguous())
+            del k, v
         else:
             for l in range(L):
                 k, v = w.prompt_kv(l, device=dev)
                 kv.prefill(l, k, v, w.queries(l, [P - 1], device=dev)[:, 0].contiguous())
                 del k, v
+        if not fullkv:
+            if ratio > 0:
+                b = kv.get_budgets()
+                row.update({"budget_rule": f"ratio {ratio}", "budget_set_by_the_rule": [int(b.min()), int(b.max())],
+                            "entries_per_head": int(b.max()) + 1})
         NS = total   # every step its own inputs: repeated keys would put exact ties into the cache
         pos = torch.arange(P, P + NS)
         lay = range(L) if not fullkv else [0] * L
@@ -460,8 +477,8 @@ def run_sweep(args):
 def run_throughput_table(args):
     """The shape of the paper's throughput table (Section 6.3) on one GPU: the 8B model shape at
     the 8K and 16K reasoning levels (9 350 and 18 700 tokens), full cache against a fixed budget of
-    1024 entries per head and against 10 % of the level (935 and 1 870), each at batch 1 and at the
-    largest batch that fits (100 GB of K/V rows, which leaves room for the prompt tensors; at most 256
+    1024 entries per head and against the ratio rule at 10 % (the library sets 935 and 1 870 per head
+    from a prompt of the level's length), each at batch 1 and at the largest batch that fits (100 GB of K/V rows, which leaves room for the prompt tensors; at most 256
     sequences per handle)."""
     wl = WORKLOADS["cfg3_llama8b"]
     dev = torch.device("cuda", 0)
@@ -470,13 +487,17 @@ def run_throughput_table(args):
     for level in (9350, 18700):
         per_seq_full = L * H * level * 512
         rows = [("full cache", None, 1), ("full cache", None, min(256, int(100e9 // per_seq_full)))]
-        for name, budget in (("fixed-1024", 1024), (f"ratio-10%-{level // 10}", level // 10)):
+        for name, budget in (("fixed-1024", 1024), ("ratio-10%", level // 10)):
             per_seq = L * H * (budget + 1) * 512
-            rows += [(name, budget, 1), (name, budget, min(256, int(100e9 // per_seq)))]
+            # (the prompt of a ratio row is the whole level: its k and v tensors, batch x level x H x 128
+            # bf16 each, must fit beside the pool while one layer is loaded)
+            cap = 256 if name != "ratio-10%" else min(256, int(10e9 // (level * H * 128 * 2 * 2)))
+            rows += [(name, budget, 1), (name, budget, min(cap, int(100e9 // per_seq)))]
         for name, budget, batch in rows:
             fullkv = budget is None
-            row = sweep_cell(wl, batch, budget or 1024, fullkv, level, 8 if fullkv else args.steps,
-                             3 if fullkv else max(args.warmup, 3), dev)
+            ratio = 0.1 if name == "ratio-10%" else 0.0
+            row = sweep_cell(wl, batch, (budget or 1024) + (64 if ratio else 0), fullkv, level, 8 if fullkv else args.steps,
+                             3 if fullkv else max(args.warmup, 3), dev, ratio=ratio)
             row.update({"level": level, "row": name, "concurrent_tokens": batch * level})
             if row.get("status") == "ok":
                 row["tokens_per_s"] = row["steps_per_s"] * batch

@@ -263,7 +263,7 @@ int crystalkv_validate(crystalkv_t* h, void* stream);
  *     crystalkv_validate there.
  *   - Every GPU on which the library is loaded holds the array (512 KiB) until the process ends.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress,
- *     with that device made current).  Make that first call before any stream capture begins.
+ *     with that device made current); later calls on that device reuse it.
  *   - All calls on one GPU, from any handle, share the array, and it keeps the previous
  *     call's contents; each call clears the part it uses on `stream` first.  Two calls whose
  *     work overlaps on the GPU (different streams, no ordering between them) race: order them.
