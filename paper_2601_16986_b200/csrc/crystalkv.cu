@@ -289,7 +289,10 @@ int join_side(crystalkv_t* h, cudaStream_t s) {
 
 // One attention launch on `s` and its follow-up (Algorithm 1 when it runs, the heads' new lengths
 // and the layer's next plan) on the internal stream.
-int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
+// chain: this launch scores the same, unchanged lists as the layer's previous launch (a window of
+// prompt queries): its attention kernel need not wait for that launch's LRFU kernel, only its own
+// LRFU kernel must run behind it.
+int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s, bool chain = false) {
   const bool track = true;   // every launch has a follow-up that uses a scratch set
   const long long k = h->kF;
   if (track) {
@@ -299,7 +302,7 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
     // A wait on the caller's stream costs several microseconds (the attention kernel behind it
     // no longer starts early), so one wait covers as many launches as the sets allow: it targets
     // the newest LRFU launch that has had two attention kernels' time to finish.
-    const long long need = std::max(k - NSETS, h->lastF[layer]);
+    const long long need = chain ? k - NSETS : std::max(k - NSETS, h->lastF[layer]);
     if (need >= 0 && need > h->joined) {
       const long long target = std::max(need, k - 3);
       CK(h, cudaStreamWaitEvent(s, h->evF[target % crystalkv::EV_RING], 0));
@@ -335,6 +338,7 @@ int launch_step(crystalkv_t* h, DecodeParams& p, int layer, cudaStream_t s) {
     p.done_ctr = h->done_ctr + 2 * si;
     CK(h, cudaEventRecord(ea, s));
     CK(h, cudaStreamWaitEvent(h->side[si], ea, 0));
+    if (chain && k > 0) CK(h, cudaStreamWaitEvent(h->side[si], h->evF[(k - 1) % crystalkv::EV_RING], 0));   // (the other internal stream)
     CK(h, lrfu_dispatch(h->G, p, h->U, h->side[si]));
     CK(h, cudaEventRecord(h->evF[k % crystalkv::EV_RING], h->side[si]));
     h->lastF[layer] = k;
@@ -618,13 +622,21 @@ static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* 
   if (evict) {
     const int passes = W > 0 ? W : 1;
     const size_t qn = (size_t)c.batch * c.n_q_heads * HD;
+    int planned_groups = -1;
     for (int i = 0; i < passes; ++i) {
       // Algorithm 1 with the query of token t: steps 1-3 for every query, step 4 (down to the
       // budget, emptied pages back to the free list) after the last one
       const int t = P - passes + i;
       const bool last = i == passes - 1;
-      rc = replan(h, layer, 1, 0, last ? 0 : t + 1, s);   // a scoring pass over the first t + 1 entries
-      if (rc) return rc;
+      // a scoring pass over the first t + 1 entries; a plan serves the passes that follow it until
+      // their heads are two groups longer (pieces take their bounds from the lengths at launch)
+      const int groups = (t + 1 + GRP - 1) / GRP;
+      const bool planned = planned_groups < 0 || groups >= planned_groups + 2;
+      if (planned) {
+        rc = replan(h, layer, 1, 0, last ? 0 : t + 1, s);
+        if (rc) return rc;
+        planned_groups = groups;
+      }
       DecodeParams p = make_params(h, layer);
       p.q = static_cast<const __nv_bfloat16*>(q) + (size_t)i * qn;
       p.k_new = p.v_new = nullptr;
@@ -634,7 +646,7 @@ static int prefill_common(crystalkv_t* h, int layer, const void* k, const void* 
       if (!last) { p.n_limit = t + 1; p.hold = 1; }
       else p.plan_append = 1;   // the layer's first decode step
       h->prev_layer = -1;       // the plan kernel ahead writes what the attention kernel reads at once
-      rc = launch_step(h, p, layer, s);
+      rc = launch_step(h, p, layer, s, i > 0);
       if (rc) return rc;
     }
     rc = join_side(h, s);
