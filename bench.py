@@ -329,11 +329,17 @@ def sweep_cell(wl, batch, budget, fullkv, context, steps, warmup, dev, ratio=0.0
     sp = C.c_void_p(stream.cuda_stream)
     P_ = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
 
+    # (pointers taken once: indexing a tensor per call costs the host more than the launch itself)
+    qp = [[P_(Q[i, l]) for l in range(L)] for i in range(NS)]
+    kp = [[P_(K[i, l]) for l in range(L)] for i in range(NS)]
+    vp = [[P_(V[i, l]) for l in range(L)] for i in range(NS)]
+    op = [P_(OUT[l]) for l in range(L)]
+
     def run(n0, n1):
         for s in range(n0, n1):
             i = s % NS
             for l in range(L):
-                rc = lib.crystalkv_decode_step(h, l, P_(Q[i, l]), P_(K[i, l]), P_(V[i, l]), P_(OUT[l]), sp)
+                rc = lib.crystalkv_decode_step(h, l, qp[i][l], kp[i][l], vp[i][l], op[l], sp)
                 if rc:
                     raise RuntimeError(f"decode_step failed: {rc}")
     run(0, warmup)
@@ -397,10 +403,15 @@ def policy_cell(wl, dev, steps, warmup, lam=None, top_p=None, evict_every=1, win
     sp = C.c_void_p(stream.cuda_stream)
     P_ = lambda t: C.c_void_p(t.data_ptr())  # noqa: E731
 
+    qp = [[P_(Q[s, l]) for l in range(L)] for s in range(Q.shape[0])]
+    kp = [[P_(K[s, l]) for l in range(L)] for s in range(Q.shape[0])]
+    vp = [[P_(V[s, l]) for l in range(L)] for s in range(Q.shape[0])]
+    op = [P_(OUT[l]) for l in range(L)]
+
     def run(n0, n1):
         for s in range(n0, n1):
             for l in range(L):
-                rc = lib.crystalkv_decode_step(h, l, P_(Q[s, l]), P_(K[s, l]), P_(V[s, l]), P_(OUT[l]), sp)
+                rc = lib.crystalkv_decode_step(h, l, qp[s][l], kp[s][l], vp[s][l], op[l], sp)
                 if rc:
                     raise RuntimeError(f"decode_step failed: {rc}")
     run(0, warmup)

@@ -16,6 +16,7 @@ constexpr int NT = NW * 32;
 constexpr int STAGES = 3;           // ring depth per warp, in pages
 constexpr int RING_BYTES = NW * STAGES * PAGE_BYTES;   // 192 KB
 constexpr int GMIN = 4;             // fewest groups a streaming warp is given
+constexpr int GLAT = 12;            // ... raised up to this many to keep a head's pieces within the eight warps of one CTA
 constexpr int QH = 8;               // query heads of a group as padded for the MMA N dimension
 constexpr int MAX_UNITS_PER_CALL = 2048;   // heads of one layer launch (bounded by the planner's shared memory)
 constexpr int NSETS = 16;           // logit scratch sets cycled by consecutive launches

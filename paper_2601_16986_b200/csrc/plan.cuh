@@ -89,7 +89,11 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
   bool packed = false;
   int* hist = red + 16;   // [32][4]: counts of two run lengths per word, 16 bits each (U < 65536)
   if (Gtot > 0 && U <= nWarps && grid * NW == nWarps && grid <= 256 && nWarps < 4096) {
-    const int T0 = max(max(1, (Gtot + nWarps - 1) / nWarps), min(GMIN, gmax));   // pieces shorter than GMIN groups
+    // A launch with few groups per warp is bound by the steps a head's result goes through, not by
+    // bytes: pieces are then made long enough (up to GLAT groups) for the longest head to stay inside
+    // one CTA, whose merge is one barrier instead of a trip through global memory.
+    const int gfloor = min(gmax, max(GMIN, min(GLAT, (gmax + NW - 1) / NW)));
+    const int T0 = max(max(1, (Gtot + nWarps - 1) / nWarps), gfloor);   // pieces shorter than GMIN groups
                                                                                 // cost more in starts and merges than they gain
     for (int round = 0; round < 4 && !packed; ++round) {
       const int Tc = T0 + round * 32 + lane;
