@@ -83,7 +83,7 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
   // ---- the piece bound T.  Heads are cut into ceil(g_u / T) pieces; the smallest T is wanted for
   // which all heads can be placed with every head's pieces inside one CTA (such a head is merged in
   // shared memory; one that straddles CTAs goes through global memory and a ticket, which costs the
-  // launch two to three microseconds at its end).  32 candidates are tried at once: warp x counts the
+  // launch several microseconds at its end).  32 candidates are tried at once: warp x counts the
   // runs of every length over the heads u = x mod 8, lane c for T0 + c; warp 0 then packs them.
   int T = 0x7fffffff;
   bool packed = false;
@@ -95,8 +95,9 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
     const int gfloor = min(gmax, max(GMIN, min(GLAT, (gmax + NW - 1) / NW)));
     const int T0 = max(max(1, (Gtot + nWarps - 1) / nWarps), gfloor);   // pieces shorter than GMIN groups
                                                                                 // cost more in starts and merges than they gain
-    for (int round = 0; round < 4 && !packed; ++round) {
-      const int Tc = T0 + round * 32 + lane;
+    // first feasible bound among Tfirst .. Tfirst + 31, or -1
+    auto first_that_packs = [&](int Tfirst) {
+      const int Tc = Tfirst + lane;
       if (tid < 128) hist[tid] = 0;
       __syncthreads();
       unsigned h4[4] = {0u, 0u, 0u, 0u};
@@ -110,7 +111,6 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
 #pragma unroll
       for (int x = 0; x < 4; ++x) atomicAdd(reinterpret_cast<unsigned*>(hist) + lane * 4 + x, h4[x]);
       __syncthreads();
-      int ok = 0;
       if (tid < 32) {
         int cnt[8];
 #pragma unroll
@@ -120,13 +120,30 @@ __device__ __forceinline__ void write_plan(const State& st, const Plan& pl, int 
           cnt[2 * x + 1] = (int)(v >> 16);
         }
         const int full = cnt[0];
-        ok = ctas_needed(full, cnt) <= grid;
+        const int ok = ctas_needed(full, cnt) <= grid;
         const unsigned m = __ballot_sync(0xffffffffu, ok);
-        if (lane == 0) red[0] = m ? T0 + round * 32 + (__ffs(m) - 1) : -1;
+        if (lane == 0) red[0] = m ? Tfirst + (__ffs(m) - 1) : -1;
       }
       __syncthreads();
-      if (red[0] > 0) { T = red[0]; packed = true; }
+      const int found = red[0];
       __syncthreads();
+      return found;
+    };
+    for (int round = 0; round < 4 && !packed; ++round) {
+      const int found = first_that_packs(T0 + round * 32);
+      if (found > 0) { T = found; packed = true; }
+    }
+    // Heads of more than eight pieces go through global memory, which costs the end of the launch
+    // about as much as seven groups of streaming.  When pieces long enough for the longest head to fit
+    // one CTA (gmax / 8 groups) cost less than that -- streaming is bound by the longer of a warp's own
+    // groups and its share of the HBM rate, 7/4 group times per group at full occupancy -- they are taken.
+    const int Tb = (gmax + NW - 1) / NW;
+    if (packed && Tb > T) {
+      const int hbm = (int)(((long long)Gtot * 7 / 4 + nWarps - 1) / nWarps);
+      if (Tb <= max(T, hbm) + 7) {
+        const int found = first_that_packs(Tb);
+        if (found > 0 && found <= Tb + 2) T = found;
+      }
     }
   }
   if (!packed && Gtot > 0 && U <= nWarps) {
