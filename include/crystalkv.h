@@ -297,6 +297,15 @@ int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, in
 int crystalkv_debug_get_plan(crystalkv_t* h, int layer, int32_t* hdr_host, int32_t* wrange_host,
                              int32_t warps_cap, int32_t* desc_host, int32_t pieces_cap, void* stream);
 
+/*
+ * Test hook for the launch planner's counting rule (the paper has no counterpart; needs no GPU
+ * and no handle): the number of CTAs of eight warps that hold `whole_ctas` CTAs taken whole plus
+ * runs_by_length[s] runs of s consecutive warps, s = 1 .. 7 (entry 0 is ignored; host int32[8]),
+ * when the runs are placed longest first, each into the open CTA with the fewest free warps that
+ * still holds it.  Returns that count (>= 0), or EINVAL for a NULL array or a negative entry.
+ */
+int crystalkv_debug_ctas_needed(int32_t whole_ctas, const int32_t* runs_by_length);
+
 const char* crystalkv_strerror(int code);
 const char* crystalkv_last_error(crystalkv_t* h);
 

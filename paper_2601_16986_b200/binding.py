@@ -101,6 +101,7 @@ def load_library():
     lib.crystalkv_validate_static.argtypes = [vp, vp, vp]
     lib.crystalkv_debug_set_page.argtypes = [vp, i32, i32, i32, C.c_int32, C.c_int32, vp]
     lib.crystalkv_debug_get_plan.argtypes = [vp, i32, vp, vp, C.c_int32, vp, C.c_int32, vp]
+    lib.crystalkv_debug_ctas_needed.argtypes = [C.c_int32, vp]
     lib.crystalkv_strerror.argtypes = [i32]
     lib.crystalkv_strerror.restype = C.c_char_p
     lib.crystalkv_last_error.argtypes = [vp]

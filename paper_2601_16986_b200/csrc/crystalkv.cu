@@ -1063,6 +1063,16 @@ int crystalkv_debug_set_page(crystalkv_t* h, int layer, int seq, int kv_head, in
   return CRYSTALKV_OK;
 }
 
+int crystalkv_debug_ctas_needed(int32_t whole_ctas, const int32_t* runs_by_length) {
+  if (!runs_by_length || whole_ctas < 0) return CRYSTALKV_EINVAL;
+  int cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  for (int s = 1; s < 8; ++s) {
+    if (runs_by_length[s] < 0) return CRYSTALKV_EINVAL;
+    cnt[s] = runs_by_length[s];
+  }
+  return ctas_needed(whole_ctas, cnt);
+}
+
 int crystalkv_debug_get_plan(crystalkv_t* h, int layer, int32_t* hdr_host, int32_t* wrange_host, int32_t warps_cap,
                              int32_t* desc_host, int32_t pieces_cap, void* stream) {
   if (!h) return CRYSTALKV_EINVAL;

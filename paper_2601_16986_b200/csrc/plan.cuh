@@ -22,7 +22,7 @@ namespace ckv {
 // warps that still holds it, so a CTA with c free warps takes c / s runs of length s one after the
 // other: the loop below moves whole classes of CTAs at once and counts exactly what the
 // run-by-run placement in write_plan() does.
-__device__ __forceinline__ int ctas_needed(int full, const int (&cnt)[8]) {
+__host__ __device__ __forceinline__ int ctas_needed(int full, const int (&cnt)[8]) {
   int open[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // open[c]: CTAs with c free warps
   int ctas = full;
 #pragma unroll
@@ -32,7 +32,7 @@ __device__ __forceinline__ int ctas_needed(int full, const int (&cnt)[8]) {
     for (int c = s; c <= 8; ++c) {
       const int q = c / s;                              // runs one such CTA takes
       const int have = (c == 8) ? (n + q - 1) / q : open[c];   // fresh CTAs are not counted in open[]
-      const int nb = min(have, n / q);                  // CTAs filled with q runs
+      const int nb = have < n / q ? have : n / q;       // CTAs filled with q runs
       int left = c - q * s;
       if (c == 8) ctas += nb; else open[c] -= nb;
       open[left] += nb;

@@ -62,3 +62,43 @@ def test_binding_refuses_to_run_without_a_gpu():
         pytest.skip("a GPU is present")
     with pytest.raises(CrystalKVError):
         CrystalKV(Config(n_layers=1, n_q_heads=2, n_kv_heads=1, batch=1, budget_per_head=8, max_context=32))
+
+
+def _place_runs_one_by_one(whole, runs):
+    """Best fit, longest first, one run at a time: the placement the planner performs."""
+    free = []            # free warps of every open CTA
+    for s in range(7, 0, -1):
+        for _ in range(runs[s]):
+            fits = [c for c in free if c >= s]
+            if fits:
+                c = min(fits)
+                free.remove(c)
+            else:
+                c = 8
+            if c - s:
+                free.append(c - s)
+            if c == 8:
+                whole += 1   # a CTA was opened
+    return whole
+
+
+def test_the_planners_count_equals_placing_the_runs_one_by_one(lib):
+    """The launch planner counts the CTAs a placement needs by moving whole classes of CTAs at
+    once; the placement itself goes run by run.  The two must agree for every mix of run lengths,
+    or a plan could be chosen that then does not fit the grid."""
+    import numpy as np
+    rng = np.random.default_rng(7)
+    cases = [[0] * 8, [0, 1, 0, 0, 0, 0, 0, 0], [0, 0, 0, 0, 0, 0, 0, 5], [0, 9, 0, 0, 0, 0, 0, 3],
+             [0, 0, 4, 0, 0, 0, 2, 0], [0, 3, 3, 3, 3, 3, 3, 3]]
+    for _ in range(400):
+        top = int(rng.integers(1, 40))
+        cases.append([0] + [int(x) for x in rng.integers(0, top, size=7)])
+    for runs in cases:
+        arr = (C.c_int32 * 8)(*runs)
+        for whole in (0, 3):
+            got = lib.crystalkv_debug_ctas_needed(whole, arr)
+            assert got == _place_runs_one_by_one(whole, runs), (whole, runs, got)
+    assert lib.crystalkv_debug_ctas_needed(0, None) == -1
+    bad = (C.c_int32 * 8)(0, -1, 0, 0, 0, 0, 0, 0)
+    assert lib.crystalkv_debug_ctas_needed(0, bad) == -1
+    assert lib.crystalkv_debug_ctas_needed(-1, (C.c_int32 * 8)()) == -1
