@@ -9,9 +9,13 @@
 // (the copies only need the cache, not the queries), waits for a stage on its mbarrier, and runs
 // both contractions on the tensor cores with keys on the MMA M dimension and the (padded) query
 // heads on N = 8:   S[16 keys x 8 heads] = K Q^T,   O^T[128 x 8 heads] += V^T P^T.
-// A head that is one piece is written out directly; otherwise every piece publishes its
-// (m, l, O) partial and the warp whose partial completes the head merges them into `out` (after
-// its own pieces, if it has more).  The arriving token is written into the head's hole (the place
+// A head that is one piece is written out directly.  A head whose pieces sit in consecutive warps
+// of this CTA (the plan arranges that and marks it) is merged in shared memory: every warp leaves
+// its (m, l, O) partial in its idle ring stages, the head's warps meet at a named barrier and
+// share the query heads.  A head of more than eight pieces is merged that way run by run (whole
+// CTAs and one shorter run) and its runs' partials through global memory: the warp whose ticket
+// completes the head merges them into `out`; so is a head that the plan could not keep together
+// (after the warp's own pieces, if it has more).  The arriving token is written into the head's hole (the place
 // an evicted entry left, or the end of the list) by the warp that streams that group.  The scaled
 // logits of the step are left in the scratch for the LRFU kernel, which marks hits from the final
 // softmax weights without reading the cache again; the lines of the metadata that kernel will

@@ -13,7 +13,8 @@
 //            within its budget; the place of a single leaver becomes the head's hole, which
 //            the next arriving token fills: nothing is moved.
 // A launch without Algorithm 1 (answer stage, full-cache mode) only lets every head keep its new
-// entry.  Either way the CTA that finishes last writes the layer's next launch plan (plan.cuh).
+// entry.  Either way the CTA that finishes last writes the layer's next launch plan (plan.cuh) when
+// a head's length has drifted from the one the current plan was made for.
 // The mass walk uses 2^-40 fixed-point integers so it is exact and order independent; the
 // threshold is relative to the integer total, so a common factor on pbar changes nothing.
 #pragma once

@@ -1,16 +1,17 @@
 // Launch plan of a layer's attention kernel: which warp streams which groups of which head.
 //
-// Every head is cut into pieces of nearly equal length, at most T groups (pages of 16 keys)
-// each, with T the smallest bound for which the pieces of all heads fit the grid's warps: one
-// piece per warp, no warp with more than T groups, whatever the heads' lengths are (after the
-// budgets have been reallocated heads hold a few hundred to a few thousand entries).  Pieces go
-// round the SMs one by one, so every SM streams the same number of them to within one.  With
-// more heads than warps every head is one piece and a warp takes several in turn.  A head of
-// several pieces is merged from their partial results.  The plan only depends on the heads'
-// lengths, so it is written by whichever kernel changed them (the LRFU kernel of the layer's
-// previous step once a head has drifted from the planned length, the shrink pass of a
-// reallocation, the prompt insertion) and the attention kernel starts streaming without deriving
-// anything but its pieces' bounds from the heads' current lengths.
+// Every head is cut into k = ceil(g / T) pieces of nearly equal length, at most T groups (pages of
+// 16 keys) each, one piece per warp, and all pieces of a head are placed in consecutive warps of
+// ONE CTA, where the head is merged in shared memory (a head of more than eight pieces takes whole
+// CTAs and one shorter run).  T is the smallest bound for which such a placement fits the grid,
+// whatever the heads' lengths are (after the budgets have been reallocated heads hold a few hundred
+// to a few thousand entries); longer pieces are taken where they keep heads inside one CTA at less
+// cost than the merge through global memory they avoid.  With more heads than warps every head is
+// one piece and a warp takes several in turn.  The plan only depends on the heads' lengths, so it
+// is written by whichever kernel changed them (the LRFU kernel of the layer's previous step once a
+// head has drifted from the planned length, the shrink pass of a reallocation, the prompt
+// insertion) and the attention kernel starts streaming without deriving anything but its pieces'
+// bounds from the heads' current lengths.
 #pragma once
 #include "common.cuh"
 
