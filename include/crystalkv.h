@@ -2,9 +2,9 @@
  * crystalkv.h — C ABI of the Crystal-KV decode hot path for NVIDIA B200 (sm_100a).
  *
  * One handle owns, on one GPU, the compressed KV cache of `batch` independent
- * sequences of a GQA transformer: a slot-indexed K/V pool per sequence, per
- * (sequence, layer, kv head) slot lists with CRF / last-hit-time metadata, and the
- * per-head budgets.  Notation follows the paper: B budget, p top-p threshold, lambda
+ * sequences of a GQA transformer: a pool of K/V pages (16 entries each) per sequence,
+ * per (sequence, layer, kv head) a page table and the entries' CRF / last-hit-time
+ * metadata, and the per-head budgets.  Notation follows the paper: B budget, p top-p threshold, lambda
  * CRF decay, t time step, tau last hit time, CRF the combined recency-frequency score.
  *
  * Conventions
@@ -123,7 +123,8 @@ int crystalkv_prefill_window(crystalkv_t* h, int layer, const void* k, const voi
  * Algorithm 1): appends (k_new, v_new) at time t = previous t + 1, attends the G
  * queries of every kv head over its cache, writes `out`, and in the think stage of
  * evict mode marks the top-p hit entries, updates CRF/tau (steps 2-3) and evicts the
- * lowest-CRF entry of every head that is over budget (step 4), reusing its slot.
+ * lowest-CRF entry of every head that is over budget (step 4); the next arriving token
+ * takes its place.
  *   q, out dev [batch][Hq][128]        k_new, v_new dev [batch][H][128]
  * Errors: EINVAL; ESTATE before prefill or when t would reach max_context or a head
  * would outgrow its capacity.
@@ -162,8 +163,8 @@ int crystalkv_set_stage(crystalkv_t* h, int stage);
 /*
  * Algorithm 2 (Section 5.3), per sequence: aggregates every head's CRF decayed to the
  * time of the last step, recomputes integer budgets that sum to B_total, and makes
- * heads whose budget shrank evict down to it; freed slots return to the sequence's
- * free list for heads that grew.  All layers must be at the same time step.
+ * heads whose budget shrank evict down to it; the pages they no longer need return to the
+ * sequence's free list for heads that grew.  All layers must be at the same time step.
  * Errors: ESTATE (layers out of step, FullKV mode, before prefill).
  */
 int crystalkv_rebudget(crystalkv_t* h, void* stream);

@@ -275,7 +275,7 @@ class CrystalKV:
 
     def validate_static(self) -> np.ndarray:
         """The same check without any device allocation (scratch built into the library; at
-        most 2**17 pool pages).  Returns int32[2]: ids out of range, slots not owned once."""
+        most 2**17 pool pages).  Returns int32[2]: page ids out of range, pages not owned exactly once."""
         counts = np.full(2, -1, dtype=np.int32)
         self._ck(self.lib.crystalkv_validate_static(self._h, counts.ctypes.data_as(C.c_void_p), _stream()))
         return counts
