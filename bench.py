@@ -725,7 +725,7 @@ def main():
         prep_in.fill(args.warmup)          # the timed steps' inputs are resident before the region starts (Ku <= 20 < 64)
         ms_u, roofline_uniform = timed_region(args.warmup, s_uni, prep_in)
         roofline_uniform.update({"steps": n_uni, "ms_per_step": ms_u / n_uni, "value": world * n_uni / (ms_u / 1000.0),
-                                 "state": "fresh after the prefill: every head at the uniform budget"})
+                                 "state": "fresh after the prefill: heads of equal length (the uniform budget, or the prompt where it is shorter)"})
     for s in range(s_uni, s_prep):
         one_step(s, prep_in, False)
     barrier()
