@@ -458,7 +458,14 @@ int crystalkv_create(const crystalkv_config_t* cfg, crystalkv_t** out) {
   CKC(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, attn_kernel, NT, h->smem));
   if (bps < 1) { h->err = "attention kernel does not fit on an SM"; CREATE_FAIL(CRYSTALKV_ECUDA); }
   h->grid = h->num_sms * bps;
-  for (cudaStream_t& x : h->side) CKC(cudaStreamCreateWithFlags(&x, cudaStreamNonBlocking));
+  {
+    // The LRFU kernels run at the highest stream priority: the attention kernel of the layer after
+    // next is already queued when one of them becomes ready (it was released early and waits for
+    // shared memory), and at equal priority its CTAs, which cannot be placed yet, are served first.
+    int least = 0, greatest = 0;
+    CKC(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+    for (cudaStream_t& x : h->side) CKC(cudaStreamCreateWithPriority(&x, cudaStreamNonBlocking, greatest));
+  }
   CKC(cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking));
   CKC(cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking));
   for (int i = 0; i < crystalkv::HOST_RING; ++i) {
