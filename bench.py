@@ -13,6 +13,7 @@ workload: the 14B-shaped configuration (48 layers, 40 q / 8 kv heads, batch 32, 
 from __future__ import annotations
 
 import argparse
+import atexit
 import ctypes as C
 import json
 import os
@@ -108,8 +109,9 @@ except Exception:
 mx = nv.nvmlDeviceGetMaxClockInfo(hd, nv.NVML_CLOCK_SM)
 bits = (0x8, 0x40, 0x20, 0x4)
 print("ready", flush=True)
-i, mw = 0, 0
-while True:
+import os
+i, mw, parent, born = 0, 0, os.getppid(), time.time()
+while os.getppid() == parent and time.time() - born < 900:   # never outlives the run it samples
     sm = nv.nvmlDeviceGetClockInfo(hd, nv.NVML_CLOCK_SM)
     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(hd)
     if i % 8 == 0:
@@ -737,6 +739,7 @@ def main():
 
     # ---- warm-up and the timed steps, inputs resident before the region starts
     clk = ClockSampler(local)
+    atexit.register(clk._kill)   # (also when a step raises)
     main_in = StepInputs(n_all - s_prep)
     main_in.fill(s_prep)
     barrier()
